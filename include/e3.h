@@ -1,0 +1,198 @@
+/*
+ * e3 -- vocabulary-side hot path of entropy-holding RL for LLMs, for NVIDIA B200 (sm_100a).
+ *
+ * One C ABI, plain pointers and sizes.  Every rollout token and every training
+ * token passes through a per-row temperature softmax over the vocabulary; this
+ * library computes, in one streaming pass over the logits,
+ *   - the Shannon entropy of softmax(z / tau)               (paper: Eq. "entropy", App. A)
+ *   - the log-probability of a given or a sampled token     (Sec. 3.1, importance ratio)
+ *   - a reproducible Gumbel-max sample                      (Sec. 2 / Sec. 5.1: tokens are drawn from softmax(z/tau))
+ * plus the masked mean entropy that drives the temperature scheduler (Sec. 4.2),
+ * the group-relative advantage (Eq. "adv") over ragged rollout groups, and two
+ * tiny host functions: Algorithm 1 (rollout budget) and Eq. "tp_adj" with annealing.
+ *
+ * Conventions for every device call
+ *   - "device" pointers are CUDA device pointers owned by the caller; the
+ *     library allocates and frees nothing and keeps no state between calls.
+ *   - Work is enqueued on `stream` (a cudaStream_t passed as void*; NULL = the
+ *     legacy default stream).  Calls never synchronise, print or abort.
+ *   - The return value reports what the host can see (bad sizes, NULL
+ *     pointers, launch failure).  Problems only the device can see (NaN or
+ *     +inf logit, a row of -inf only, tau < 0 or not finite) mark that row:
+ *     token -1, log-prob and entropy NaN.  Other rows are unaffected.
+ *   - Results are bit-reproducible for identical arguments.
+ *   - rows == 0 / n == 0 / n_groups == 0 are valid no-ops.
+ */
+#ifndef E3_H_
+#define E3_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define E3_API __attribute__((visibility("default")))
+#else
+#define E3_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  E3_OK = 0,
+  E3_ERR_INVALID_ARG = 1, /* NULL required pointer, negative size, V < 1 or V >= 2^31, row_stride < V, ... */
+  E3_ERR_DTYPE = 2,       /* dtype is neither E3_F32 nor E3_BF16 */
+  E3_ERR_ALIGNMENT = 3,   /* a pointer is not aligned to its element type */
+  E3_ERR_WORKSPACE = 4,   /* workspace missing or smaller than e3_workspace_bytes() says */
+  E3_ERR_INFEASIBLE = 5,  /* Algorithm 1: needs G_min <= G <= G_max */
+  E3_ERR_CUDA = 6,        /* a CUDA runtime call failed (no device, launch error) */
+  E3_ERR_TIMEOUT = 7      /* reserved: a bounded device-side wait ran out */
+} e3_status;
+
+typedef enum { E3_F32 = 0, E3_BF16 = 1 } e3_dtype;
+
+/* Sampler of e3_sample.  Both draw exactly from softmax(z / tau) up to the
+ * resolution of their uniforms (2^-40 and 2^-32). */
+typedef enum {
+  E3_SAMPLER_TOKEN = 0, /* one Gumbel per vocabulary entry: tok = argmax_i (z_i/tau + g_i) */
+  E3_SAMPLER_BLOCK = 1  /* one Gumbel per block of E3_SAMPLE_BLOCK consecutive entries applied to the
+                           block's log-sum-exp, then inverse CDF inside the winning block */
+} e3_sampler;
+#define E3_SAMPLE_BLOCK 256
+
+typedef enum {
+  E3_CALL_SAMPLE = 0,
+  E3_CALL_TOKEN_LOGP_ENTROPY = 1,
+  E3_CALL_MASKED_MEAN_ENTROPY = 2
+} e3_call;
+
+/* Human-readable name of a status code (static string). */
+E3_API const char *e3_status_string(e3_status s);
+
+/* Bytes of device scratch a call needs for the given problem size (0 = none;
+ * the call then accepts workspace == NULL).  For E3_CALL_MASKED_MEAN_ENTROPY
+ * `rows` is the number of tokens n and V, dt are ignored. */
+E3_API size_t e3_workspace_bytes(e3_call which, int64_t rows, int64_t V, e3_dtype dt);
+
+/*
+ * Rollout step.  For every row r: p = softmax(logits[r, 0..V) / temps[r])
+ * (App. A); out_ent[r] = -sum p ln p (Eq. "entropy"); out_tok[r] = one token
+ * drawn from p with the Gumbel-max construction; out_logp[r] = ln p[out_tok[r]].
+ *
+ *   logits      device, row-major [rows, V], element type `dt`, row r starts at
+ *               element r * row_stride (row_stride >= V, in elements).  Rows whose
+ *               start is 16-byte aligned take the vectorised path; others a slower one.
+ *   temps       device float [rows].  tau > 0 samples; tau == 0 is greedy
+ *               (lowest-index arg-max, logp = 0, ent = 0); tau < 0, NaN, inf mark the row invalid.
+ *   seed, counter, row_base
+ *               the draw is a pure function of (seed, counter, row_base + r, vocabulary index):
+ *               Philox4x32-10 with key = seed and counter words
+ *               (call index, row_base + r, counter low word, counter high bits << 8 | stream tag).
+ *               counter < 2^56: the decode step; row_base: index of this call's first row in the
+ *               whole batch, so that a batch split over several calls or devices draws the same tokens.
+ *               Sampler 0: u_i = (c_i + (x_i + 1/2) 2^-32) / 256 with c_i byte (i mod 16) of call i/16 of
+ *               stream 0 and x_i word (i mod 4) of call i/4 of stream 1; g_i = -ln(-ln u_i);
+ *               ties go to the lower index.
+ *               Sampler 1: u_b = (x_b + 1/2) 2^-32, x_b word (b mod 4) of call b/4 of stream 2, for block b;
+ *               the in-block draw uses word 0 of call 0 of stream 3.
+ *   out_tok     device int32 [rows], required.   out_logp, out_ent: device float [rows], each may be NULL.
+ *   workspace   device scratch of e3_workspace_bytes(E3_CALL_SAMPLE, ...) bytes (NULL when that is 0).
+ * -inf logits are allowed (probability 0, never drawn).
+ */
+E3_API e3_status e3_sample(const void *logits, e3_dtype dt, int64_t rows, int64_t V, int64_t row_stride,
+                    const float *temps, uint64_t seed, uint64_t counter, int64_t row_base, e3_sampler sampler,
+                    int32_t *out_tok, float *out_logp, float *out_ent,
+                    void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * Training-side pass.  For every row with mask[r] != 0:
+ * out_logp[r] = ln softmax(logits[r] / tau_r)[targets[r]], out_ent[r] = entropy of that
+ * distribution.  The paper divides the logits by the sampling temperature in the training
+ * forward as well (Sec. 4.2), so the call takes tau: temps[r] when temps != NULL, else temp_scalar.
+ * Here tau must be > 0 and finite.  Rows with mask[r] == 0 get 0 in both outputs and their
+ * logits are not read.  A target outside [0, V) gives out_logp = NaN (entropy still valid).
+ *
+ *   targets     device int32 [rows];  mask: device uint8 [rows] or NULL (= all ones)
+ *   out_logp, out_ent   device float [rows], each may be NULL
+ * Other arguments as in e3_sample.
+ */
+E3_API e3_status e3_token_logp_entropy(const void *logits, e3_dtype dt, int64_t rows, int64_t V, int64_t row_stride,
+                                const int32_t *targets, const uint8_t *mask,
+                                const float *temps, float temp_scalar,
+                                float *out_logp, float *out_ent,
+                                void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * Batch entropy H_t of the scheduler (Sec. 4.2: "average entropy" of a batch), read as the mean
+ * over all response tokens: out_mean = sum_j mask[j] ent[j] / sum_j mask[j], accumulated in
+ * fp64 in a fixed order.  out_count = sum_j mask[j].  count == 0 gives mean NaN.
+ *
+ *   ent         device float [n];  mask: device uint8 [n] or NULL (= all ones)
+ *   out_mean, out_count   device double scalars, required
+ *   workspace   device scratch of e3_workspace_bytes(E3_CALL_MASKED_MEAN_ENTROPY, n, 0, 0) bytes;
+ *               contents on entry do not matter.
+ */
+E3_API e3_status e3_masked_mean_entropy(const float *ent, const uint8_t *mask, int64_t n,
+                                 double *out_mean, double *out_count,
+                                 void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * Group-relative advantage (Eq. "adv"): inside each rollout group g = rows
+ * [group_offsets[g], group_offsets[g+1]):  A_i = (r_i - mean) / (std + eps).
+ * Groups may have any size (the rollout budget of Algorithm 1 makes them ragged).
+ * std is the sample standard deviation (divide by n-1) when unbiased != 0, else the population one.
+ * eps > 0 makes a group with identical rewards give exactly 0, as Sec. 4.2 assumes.
+ * A group of one gives 0; an empty group writes nothing.
+ *
+ *   rewards        device float [group_offsets[n_groups]]
+ *   group_offsets  device int64 [n_groups + 1], non-decreasing, [0] == 0
+ *   out_adv        device float, same length as rewards
+ *   out_group_flags  NULL or device uint8 [n_groups]: bit 0 = all rewards equal, bit 1 = all rewards zero
+ */
+E3_API e3_status e3_group_advantage(const float *rewards, const int64_t *group_offsets, int64_t n_groups,
+                             float eps, int unbiased, float *out_adv, uint8_t *out_group_flags, void *stream);
+
+/*
+ * Algorithm 1 (Dynamic Rollout Budget), host only.  k[i] in [0, 1] is the normalised difficulty
+ * rank of question i; out_G[i] receives its rollout count with sum out_G = B * G and
+ * G_min <= out_G[i] <= G_max.  Steps as printed: start at G_min, add floor(N_rem k_i / sum k)
+ * (capped at G_max), hand the remainder out in descending order of k (ties: lower index first).
+ * greedy_mode 0 fills each question to G_max in turn; 1 gives one rollout per question per sweep.
+ * sum k == 0 gives every question G.  All pointers are host pointers.
+ * Errors: E3_ERR_INFEASIBLE unless G_min <= G <= G_max; E3_ERR_INVALID_ARG for k outside [0,1] or NaN.
+ */
+E3_API e3_status e3_allocate_budget(const double *k, int64_t B, int32_t G, int32_t G_min, int32_t G_max,
+                             int greedy_mode, int32_t *out_G);
+
+/* Scheduler state, owned by the caller; plain data, can be copied or stored as is. */
+typedef struct {
+  double tau;      /* current temperature tau_t (> 0) */
+  double H_init;   /* entropy level to hold; NaN or <= 0 = not recorded yet */
+  int64_t t;       /* training step, advanced by every successful update */
+  int64_t t_anneal;/* first step of the annealing phase */
+  int64_t t_max;   /* last training step; t_max <= t_anneal switches annealing off */
+  double eta;      /* annealing floor: target entropy goes from H_init to eta * H_init */
+  int64_t V;       /* vocabulary size |V| in Eq. "tp_adj" (>= 3) */
+  double tau_min;  /* clamp, used when tau_max > 0 */
+  double tau_max;
+} e3_sched;
+
+/*
+ * Temperature scheduler (Eq. "tp_adj" and the annealing equation, Sec. 4.2), host only:
+ *   alpha = H_target / H_t,  tau_{t+1} = tau_t (1 + tau_t ln(alpha) / (ln|V| + ln ln|V|)),
+ *   H_target = H_init for t < t_anneal, else
+ *              H_init [eta + (1 - eta) (1/2) (1 + cos(pi (t - t_anneal) / (t_max - t_anneal)))].
+ * The first call with H_init unset records H_init = H_t and keeps tau.  On success the state is
+ * updated (tau, t) and *tau_next = tau.  H_t <= 0 or not finite, tau <= 0, V < 3, or an update that
+ * would leave tau <= 0 return E3_ERR_INVALID_ARG and change nothing.
+ */
+E3_API e3_status e3_update_temperature(e3_sched *s, double H_t, double *tau_next);
+
+/* Target entropy the scheduler holds at step s->t (H_init before annealing starts). */
+E3_API double e3_anneal_target(const e3_sched *s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* E3_H_ */

@@ -1,0 +1,228 @@
+"""Thin ctypes binding of ``libe3.so`` (declared in ``include/e3.h``).
+
+Argument marshalling only: every step of the path runs in the CUDA library.  Device calls take
+``torch`` CUDA tensors (used for their memory and stream, nothing else), pass raw pointers and
+sizes through the C ABI and return the output tensors.  There is no CPU fallback: if the library
+has not been built, or a tensor is not on a CUDA device, the call raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libe3.so")
+
+E3_OK = 0
+E3_F32, E3_BF16 = 0, 1
+E3_SAMPLER_TOKEN, E3_SAMPLER_BLOCK = 0, 1
+E3_CALL_SAMPLE, E3_CALL_TOKEN_LOGP_ENTROPY, E3_CALL_MASKED_MEAN_ENTROPY = 0, 1, 2
+E3_SAMPLE_BLOCK = 256
+
+EXPORTS = ("e3_status_string", "e3_workspace_bytes", "e3_sample", "e3_token_logp_entropy",
+           "e3_masked_mean_entropy", "e3_group_advantage", "e3_allocate_budget", "e3_update_temperature",
+           "e3_anneal_target")
+
+
+class E3Error(RuntimeError):
+    def __init__(self, call: str, status: int):
+        self.status = status
+        super().__init__(f"{call} failed: {status_string(status)} ({status})")
+
+
+class e3_sched(C.Structure):
+    """Mirror of the C struct ``e3_sched``."""
+    _fields_ = [("tau", C.c_double), ("H_init", C.c_double), ("t", C.c_int64), ("t_anneal", C.c_int64),
+                ("t_max", C.c_int64), ("eta", C.c_double), ("V", C.c_int64), ("tau_min", C.c_double),
+                ("tau_max", C.c_double)]
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """The loaded library; raises if it has not been built (no fallback)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2505_18573_b200.build`")
+        L = C.CDLL(LIB_PATH)
+        L.e3_status_string.restype = C.c_char_p
+        L.e3_status_string.argtypes = [C.c_int]
+        L.e3_workspace_bytes.restype = C.c_size_t
+        L.e3_workspace_bytes.argtypes = [C.c_int, C.c_int64, C.c_int64, C.c_int]
+        L.e3_sample.restype = C.c_int
+        L.e3_sample.argtypes = [C.c_void_p, C.c_int, C.c_int64, C.c_int64, C.c_int64, C.c_void_p, C.c_uint64,
+                                C.c_uint64, C.c_int64, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                                C.c_size_t, C.c_void_p]
+        L.e3_token_logp_entropy.restype = C.c_int
+        L.e3_token_logp_entropy.argtypes = [C.c_void_p, C.c_int, C.c_int64, C.c_int64, C.c_int64, C.c_void_p,
+                                            C.c_void_p, C.c_void_p, C.c_float, C.c_void_p, C.c_void_p, C.c_void_p,
+                                            C.c_size_t, C.c_void_p]
+        L.e3_masked_mean_entropy.restype = C.c_int
+        L.e3_masked_mean_entropy.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p,
+                                             C.c_size_t, C.c_void_p]
+        L.e3_group_advantage.restype = C.c_int
+        L.e3_group_advantage.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_float, C.c_int, C.c_void_p,
+                                         C.c_void_p, C.c_void_p]
+        L.e3_allocate_budget.restype = C.c_int
+        L.e3_allocate_budget.argtypes = [C.c_void_p, C.c_int64, C.c_int32, C.c_int32, C.c_int32, C.c_int, C.c_void_p]
+        L.e3_update_temperature.restype = C.c_int
+        L.e3_update_temperature.argtypes = [C.POINTER(e3_sched), C.c_double, C.POINTER(C.c_double)]
+        L.e3_anneal_target.restype = C.c_double
+        L.e3_anneal_target.argtypes = [C.POINTER(e3_sched)]
+        _lib = L
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return lib().e3_status_string(int(status)).decode()
+
+
+def _check(call: str, status: int) -> None:
+    if status != E3_OK:
+        raise E3Error(call, status)
+
+
+def _dev(t, name: str):
+    if t is None:
+        return None
+    if not t.is_cuda:
+        raise ValueError(f"{name} must be a CUDA tensor (there is no CPU path)")
+    return t
+
+
+def _ptr(t) -> int | None:
+    return None if t is None else t.data_ptr()
+
+
+def _stream(stream) -> int:
+    s = torch.cuda.current_stream() if stream is None else stream
+    return s.cuda_stream
+
+
+def _logits_desc(logits: torch.Tensor):
+    _dev(logits, "logits")
+    if logits.dim() != 2 or (logits.shape[1] > 1 and logits.stride(1) != 1):
+        raise ValueError("logits must be 2-D with a contiguous last dimension")
+    if logits.dtype == torch.float32:
+        dt = E3_F32
+    elif logits.dtype == torch.bfloat16:
+        dt = E3_BF16
+    else:
+        raise ValueError("logits must be float32 or bfloat16")
+    rows, V = logits.shape
+    stride = logits.stride(0) if rows > 1 else max(V, logits.stride(0))
+    return dt, rows, V, stride
+
+
+def e3_workspace_bytes(which: int, rows: int, V: int = 0, dt: int = E3_F32) -> int:
+    return int(lib().e3_workspace_bytes(which, rows, V, dt))
+
+
+def e3_sample(logits, temps, seed: int, counter: int, row_base: int = 0, sampler: int = E3_SAMPLER_TOKEN,
+              out_tok=None, out_logp=None, out_ent=None, want_logp: bool = True, want_ent: bool = True,
+              stream=None):
+    """Rollout step: returns (tok int32, logp float32 | None, ent float32 | None), each [rows]."""
+    dt, rows, V, stride = _logits_desc(logits)
+    _dev(temps, "temps")
+    if temps.dtype != torch.float32 or temps.numel() != rows or not temps.is_contiguous():
+        raise ValueError("temps must be a contiguous float32 tensor with one entry per row")
+    dev = logits.device
+    if out_tok is None:
+        out_tok = torch.empty(rows, dtype=torch.int32, device=dev)
+    if out_logp is None and want_logp:
+        out_logp = torch.empty(rows, dtype=torch.float32, device=dev)
+    if out_ent is None and want_ent:
+        out_ent = torch.empty(rows, dtype=torch.float32, device=dev)
+    st = lib().e3_sample(_ptr(logits), dt, rows, V, stride, _ptr(temps), seed, counter, row_base, sampler,
+                         _ptr(out_tok), _ptr(out_logp), _ptr(out_ent), None, 0, _stream(stream))
+    _check("e3_sample", st)
+    return out_tok, out_logp, out_ent
+
+
+def e3_token_logp_entropy(logits, targets, mask=None, temps=None, temp_scalar: float = 1.0, out_logp=None,
+                          out_ent=None, stream=None):
+    """Training-side pass: returns (logp float32, ent float32), each [rows]; masked rows give 0."""
+    dt, rows, V, stride = _logits_desc(logits)
+    _dev(targets, "targets"); _dev(mask, "mask"); _dev(temps, "temps")
+    if targets.dtype != torch.int32 or targets.numel() != rows:
+        raise ValueError("targets must be int32 with one entry per row")
+    if mask is not None and (mask.dtype != torch.uint8 or mask.numel() != rows):
+        raise ValueError("mask must be uint8 with one entry per row")
+    if temps is not None and (temps.dtype != torch.float32 or temps.numel() != rows):
+        raise ValueError("temps must be float32 with one entry per row")
+    dev = logits.device
+    if out_logp is None:
+        out_logp = torch.empty(rows, dtype=torch.float32, device=dev)
+    if out_ent is None:
+        out_ent = torch.empty(rows, dtype=torch.float32, device=dev)
+    st = lib().e3_token_logp_entropy(_ptr(logits), dt, rows, V, stride, _ptr(targets), _ptr(mask), _ptr(temps),
+                                     float(temp_scalar), _ptr(out_logp), _ptr(out_ent), None, 0, _stream(stream))
+    _check("e3_token_logp_entropy", st)
+    return out_logp, out_ent
+
+
+def e3_masked_mean_entropy(ent, mask=None, out=None, workspace=None, stream=None):
+    """Returns a float64 CUDA tensor [2] = (mean, count).  No host synchronisation."""
+    _dev(ent, "ent"); _dev(mask, "mask")
+    if ent.dtype != torch.float32 or not ent.is_contiguous():
+        raise ValueError("ent must be a contiguous float32 tensor")
+    n = ent.numel()
+    if mask is not None and (mask.dtype != torch.uint8 or mask.numel() != n):
+        raise ValueError("mask must be uint8 with one entry per token")
+    if out is None:
+        out = torch.empty(2, dtype=torch.float64, device=ent.device)
+    need = e3_workspace_bytes(E3_CALL_MASKED_MEAN_ENTROPY, n)
+    if workspace is None:
+        workspace = torch.empty(need, dtype=torch.uint8, device=ent.device)
+    st = lib().e3_masked_mean_entropy(_ptr(ent), _ptr(mask), n, out.data_ptr(), out.data_ptr() + 8,
+                                      _ptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream))
+    _check("e3_masked_mean_entropy", st)
+    return out
+
+
+def e3_group_advantage(rewards, group_offsets, eps: float = 1e-6, unbiased: bool = True, out_adv=None,
+                       out_flags=None, want_flags: bool = True, stream=None):
+    """Returns (adv float32 [n], flags uint8 [n_groups] | None)."""
+    _dev(rewards, "rewards"); _dev(group_offsets, "group_offsets")
+    if rewards.dtype != torch.float32 or group_offsets.dtype != torch.int64:
+        raise ValueError("rewards must be float32 and group_offsets int64")
+    ng = group_offsets.numel() - 1
+    if out_adv is None:
+        out_adv = torch.zeros_like(rewards)
+    if out_flags is None and want_flags:
+        out_flags = torch.zeros(max(ng, 0), dtype=torch.uint8, device=rewards.device)
+    st = lib().e3_group_advantage(_ptr(rewards), _ptr(group_offsets), ng, float(eps), int(bool(unbiased)),
+                                  _ptr(out_adv), _ptr(out_flags), _stream(stream))
+    _check("e3_group_advantage", st)
+    return out_adv, out_flags
+
+
+def e3_allocate_budget(k, G: int, G_min: int, G_max: int, greedy_mode: int = 0):
+    """Algorithm 1 on the host: list of per-question rollout counts."""
+    B = len(k)
+    karr = (C.c_double * max(B, 1))(*[float(x) for x in k])
+    out = (C.c_int32 * max(B, 1))()
+    st = lib().e3_allocate_budget(karr, B, G, G_min, G_max, greedy_mode, out)
+    _check("e3_allocate_budget", st)
+    return [int(out[i]) for i in range(B)]
+
+
+def make_sched(tau: float = 1.0, H_init: float = float("nan"), t: int = 0, t_anneal: int = 1 << 62,
+               t_max: int = 1 << 62, eta: float = 0.9, V: int = 151936, tau_min: float = 0.0,
+               tau_max: float = 0.0) -> e3_sched:
+    return e3_sched(tau, H_init, t, t_anneal, t_max, eta, V, tau_min, tau_max)
+
+
+def e3_update_temperature(s: e3_sched, H_t: float) -> float:
+    out = C.c_double()
+    st = lib().e3_update_temperature(C.byref(s), float(H_t), C.byref(out))
+    _check("e3_update_temperature", st)
+    return out.value
+
+
+def e3_anneal_target(s: e3_sched) -> float:
+    return float(lib().e3_anneal_target(C.byref(s)))

@@ -1,0 +1,124 @@
+// C ABI of the device calls: argument checks, parameter marshalling, launches.
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "e3.h"
+#include "e3_rows.cuh"
+#include "e3_small.cuh"
+
+namespace {
+
+inline bool misaligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) != 0; }
+
+e3_status check_logits(const void *logits, e3_dtype dt, int64_t rows, int64_t V, int64_t row_stride) {
+  if (dt != E3_F32 && dt != E3_BF16) return E3_ERR_DTYPE;
+  if (rows < 0 || V < 1 || V >= (int64_t(1) << 31) || row_stride < V) return E3_ERR_INVALID_ARG;
+  if (rows > 0 && !logits) return E3_ERR_INVALID_ARG;
+  if (misaligned(logits, dt == E3_F32 ? 4 : 2)) return E3_ERR_ALIGNMENT;
+  return E3_OK;
+}
+
+bool rows_are_16B_aligned(const void *logits, e3_dtype dt, int64_t row_stride) {
+  const int64_t esize = dt == E3_F32 ? 4 : 2;
+  return !misaligned(logits, 16) && (row_stride * esize) % 16 == 0;
+}
+
+void philox_round_keys(uint64_t seed, uint32_t rk[20]) {
+  uint32_t k0 = static_cast<uint32_t>(seed), k1 = static_cast<uint32_t>(seed >> 32);
+  for (int r = 0; r < 10; ++r) {
+    rk[2 * r] = k0;
+    rk[2 * r + 1] = k1;
+    k0 += 0x9E3779B9u;  // Weyl increments of the Philox key schedule
+    k1 += 0xBB67AE85u;
+  }
+}
+
+}  // namespace
+
+extern "C" size_t e3_workspace_bytes(e3_call which, int64_t rows, int64_t V, e3_dtype dt) {
+  (void)V;
+  (void)dt;
+  switch (which) {
+    case E3_CALL_SAMPLE: return 0;
+    case E3_CALL_TOKEN_LOGP_ENTROPY: return 0;
+    case E3_CALL_MASKED_MEAN_ENTROPY: return e3::mean_workspace_bytes(rows < 0 ? 0 : rows);
+  }
+  return 0;
+}
+
+extern "C" e3_status e3_sample(const void *logits, e3_dtype dt, int64_t rows, int64_t V, int64_t row_stride,
+                               const float *temps, uint64_t seed, uint64_t counter, int64_t row_base,
+                               e3_sampler sampler, int32_t *out_tok, float *out_logp, float *out_ent,
+                               void *workspace, size_t workspace_bytes, void *stream) {
+  (void)workspace;
+  (void)workspace_bytes;
+  e3_status st = check_logits(logits, dt, rows, V, row_stride);
+  if (st != E3_OK) return st;
+  if (sampler != E3_SAMPLER_TOKEN && sampler != E3_SAMPLER_BLOCK) return E3_ERR_INVALID_ARG;
+  if (row_base < 0 || counter >= (uint64_t(1) << 56)) return E3_ERR_INVALID_ARG;
+  if (rows == 0) return E3_OK;
+  if (!temps || !out_tok) return E3_ERR_INVALID_ARG;
+  if (misaligned(temps, 4) || misaligned(out_tok, 4) || misaligned(out_logp, 4) || misaligned(out_ent, 4))
+    return E3_ERR_ALIGNMENT;
+
+  e3::RowsParams p = {};
+  p.logits = logits; p.rows = rows; p.V = V; p.row_stride = row_stride;
+  p.temps = temps; p.temp_scalar = 1.f;
+  p.out_tok = out_tok; p.out_logp = out_logp; p.out_ent = out_ent;
+  philox_round_keys(seed, p.round_key);
+  p.ctr_lo = static_cast<uint32_t>(counter);
+  p.ctr_hi8 = static_cast<uint32_t>(counter >> 32) << 8;
+  p.row_base = static_cast<uint32_t>(row_base);
+  p.mode = e3::kModeSample;
+  cudaError_t e = e3::launch_rows(p, static_cast<int>(dt), static_cast<int>(sampler),
+                                  rows_are_16B_aligned(logits, dt, row_stride), static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? E3_OK : E3_ERR_CUDA;
+}
+
+extern "C" e3_status e3_token_logp_entropy(const void *logits, e3_dtype dt, int64_t rows, int64_t V,
+                                           int64_t row_stride, const int32_t *targets, const uint8_t *mask,
+                                           const float *temps, float temp_scalar, float *out_logp, float *out_ent,
+                                           void *workspace, size_t workspace_bytes, void *stream) {
+  (void)workspace;
+  (void)workspace_bytes;
+  e3_status st = check_logits(logits, dt, rows, V, row_stride);
+  if (st != E3_OK) return st;
+  if (rows == 0) return E3_OK;
+  if (!targets) return E3_ERR_INVALID_ARG;
+  if (misaligned(targets, 4) || misaligned(temps, 4) || misaligned(out_logp, 4) || misaligned(out_ent, 4))
+    return E3_ERR_ALIGNMENT;
+
+  e3::RowsParams p = {};
+  p.logits = logits; p.rows = rows; p.V = V; p.row_stride = row_stride;
+  p.temps = temps; p.temp_scalar = temp_scalar;
+  p.targets = targets; p.mask = mask;
+  p.out_logp = out_logp; p.out_ent = out_ent;
+  p.mode = e3::kModeTargets;
+  cudaError_t e = e3::launch_rows(p, static_cast<int>(dt), -1, rows_are_16B_aligned(logits, dt, row_stride),
+                                  static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? E3_OK : E3_ERR_CUDA;
+}
+
+extern "C" e3_status e3_masked_mean_entropy(const float *ent, const uint8_t *mask, int64_t n, double *out_mean,
+                                            double *out_count, void *workspace, size_t workspace_bytes,
+                                            void *stream) {
+  if (n < 0 || !out_mean || !out_count || (n > 0 && !ent)) return E3_ERR_INVALID_ARG;
+  if (misaligned(ent, 4) || misaligned(out_mean, 8) || misaligned(out_count, 8) || misaligned(workspace, 8))
+    return E3_ERR_ALIGNMENT;
+  if (!workspace || workspace_bytes < e3::mean_workspace_bytes(n)) return E3_ERR_WORKSPACE;
+  cudaError_t e = e3::launch_masked_mean(ent, mask, n, out_mean, out_count, workspace,
+                                         static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? E3_OK : E3_ERR_CUDA;
+}
+
+extern "C" e3_status e3_group_advantage(const float *rewards, const int64_t *group_offsets, int64_t n_groups,
+                                        float eps, int unbiased, float *out_adv, uint8_t *out_group_flags,
+                                        void *stream) {
+  if (n_groups < 0 || !(eps >= 0.f)) return E3_ERR_INVALID_ARG;
+  if (n_groups == 0) return E3_OK;
+  if (!rewards || !group_offsets || !out_adv) return E3_ERR_INVALID_ARG;
+  if (misaligned(rewards, 4) || misaligned(group_offsets, 8) || misaligned(out_adv, 4)) return E3_ERR_ALIGNMENT;
+  cudaError_t e = e3::launch_group_advantage(rewards, group_offsets, n_groups, eps, unbiased, out_adv,
+                                             out_group_flags, static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? E3_OK : E3_ERR_CUDA;
+}

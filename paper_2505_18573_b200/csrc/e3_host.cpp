@@ -1,0 +1,102 @@
+// Host-only entry points: Algorithm 1 (Dynamic Rollout Budget) and the temperature scheduler
+// (Eq. "tp_adj" with the cosine annealing of its target entropy).  Tiny, not on the hot path.
+#include <algorithm>
+#include <cmath>
+#include <numeric>
+#include <vector>
+
+#include "e3.h"
+
+extern "C" const char *e3_status_string(e3_status s) {
+  switch (s) {
+    case E3_OK: return "E3_OK";
+    case E3_ERR_INVALID_ARG: return "E3_ERR_INVALID_ARG";
+    case E3_ERR_DTYPE: return "E3_ERR_DTYPE";
+    case E3_ERR_ALIGNMENT: return "E3_ERR_ALIGNMENT";
+    case E3_ERR_WORKSPACE: return "E3_ERR_WORKSPACE";
+    case E3_ERR_INFEASIBLE: return "E3_ERR_INFEASIBLE";
+    case E3_ERR_CUDA: return "E3_ERR_CUDA";
+    case E3_ERR_TIMEOUT: return "E3_ERR_TIMEOUT";
+  }
+  return "E3_ERR_UNKNOWN";
+}
+
+extern "C" e3_status e3_allocate_budget(const double *k, int64_t B, int32_t G, int32_t G_min, int32_t G_max,
+                                        int greedy_mode, int32_t *out_G) {
+  if (B < 0 || G_min < 0 || (B > 0 && (!k || !out_G)) || (greedy_mode != 0 && greedy_mode != 1))
+    return E3_ERR_INVALID_ARG;
+  if (G_min > G || G > G_max) return E3_ERR_INFEASIBLE;
+  for (int64_t i = 0; i < B; ++i)
+    if (!(k[i] >= 0.0 && k[i] <= 1.0)) return E3_ERR_INVALID_ARG;
+  if (B == 0) return E3_OK;
+
+  const double k_total = std::accumulate(k, k + B, 0.0);
+  if (k_total == 0.0) {
+    std::fill(out_G, out_G + B, G);
+    return E3_OK;
+  }
+  const int64_t budget = B * static_cast<int64_t>(G);
+  const int64_t spare = budget - B * static_cast<int64_t>(G_min);  // N_rem after the G_min floor
+  int64_t handed = 0;
+  for (int64_t i = 0; i < B; ++i) {
+    const int64_t share = static_cast<int64_t>(std::floor(static_cast<double>(spare) * (k[i] / k_total)));
+    const int64_t g = std::min<int64_t>(G_max, static_cast<int64_t>(G_min) + share);
+    out_G[i] = static_cast<int32_t>(g);
+    handed += g;
+  }
+  int64_t left = budget - handed;
+
+  // hardest first; equal difficulty keeps batch order
+  std::vector<int64_t> by_difficulty(B);
+  std::iota(by_difficulty.begin(), by_difficulty.end(), int64_t{0});
+  std::stable_sort(by_difficulty.begin(), by_difficulty.end(), [k](int64_t a, int64_t b) { return k[a] > k[b]; });
+
+  if (greedy_mode == 0) {
+    for (int64_t q : by_difficulty) {
+      if (left == 0) break;
+      const int64_t give = std::min<int64_t>(left, G_max - out_G[q]);
+      out_G[q] += static_cast<int32_t>(give);
+      left -= give;
+    }
+  } else {
+    bool progress = true;
+    while (left > 0 && progress) {
+      progress = false;
+      for (int64_t q : by_difficulty) {
+        if (left == 0) break;
+        if (out_G[q] < G_max) { ++out_G[q]; --left; progress = true; }
+      }
+    }
+  }
+  return left == 0 ? E3_OK : E3_ERR_INFEASIBLE;
+}
+
+extern "C" double e3_anneal_target(const e3_sched *s) {
+  if (!s) return std::nan("");
+  if (s->t < s->t_anneal || s->t_max <= s->t_anneal) return s->H_init;
+  const double progress =
+      std::min(1.0, static_cast<double>(s->t - s->t_anneal) / static_cast<double>(s->t_max - s->t_anneal));
+  const double cosine = 0.5 * (1.0 + std::cos(3.14159265358979323846 * progress));
+  return s->H_init * (s->eta + (1.0 - s->eta) * cosine);
+}
+
+extern "C" e3_status e3_update_temperature(e3_sched *s, double H_t, double *tau_next) {
+  if (!s || !tau_next) return E3_ERR_INVALID_ARG;
+  if (!std::isfinite(H_t) || H_t <= 0.0 || s->V < 3 || !(s->tau > 0.0) || !std::isfinite(s->tau))
+    return E3_ERR_INVALID_ARG;
+  if (!(s->H_init > 0.0)) {  // first batch: remember the level to hold
+    s->H_init = H_t;
+    s->t += 1;
+    *tau_next = s->tau;
+    return E3_OK;
+  }
+  const double alpha = e3_anneal_target(s) / H_t;
+  const double ln_v = std::log(static_cast<double>(s->V));
+  double tau = s->tau * (1.0 + s->tau * std::log(alpha) / (ln_v + std::log(ln_v)));
+  if (!(tau > 0.0)) return E3_ERR_INVALID_ARG;
+  if (s->tau_max > 0.0) tau = std::min(std::max(tau, s->tau_min), s->tau_max);
+  s->tau = tau;
+  s->t += 1;
+  *tau_next = tau;
+  return E3_OK;
+}

@@ -1,0 +1,120 @@
+"""CPU-side checks of the C-ABI library: it loads, exports every symbol the header declares,
+and its host entry points (Algorithm 1, temperature scheduler) agree with the oracle.
+No device call is made here."""
+import ctypes as C
+import math
+import os
+import re
+
+import numpy as np
+import pytest
+
+import oracle
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def e3():
+    from paper_2505_18573_b200 import build, binding
+    build.build()
+    binding.lib()
+    return binding
+
+
+def test_library_exports_every_declared_symbol(e3):
+    header = open(os.path.join(ROOT, "include", "e3.h")).read()
+    declared = set(re.findall(r"E3_API[^;(]*?\b(e3_\w+)\s*\(", header))
+    assert declared == set(e3.EXPORTS)
+    L = C.CDLL(e3.LIB_PATH)
+    for name in declared:
+        assert hasattr(L, name), name
+
+
+def test_status_strings_and_workspace(e3):
+    assert e3.status_string(0) == "E3_OK"
+    assert e3.status_string(5) == "E3_ERR_INFEASIBLE"
+    assert e3.e3_workspace_bytes(e3.E3_CALL_SAMPLE, 512, 151936, e3.E3_BF16) == 0
+    assert e3.e3_workspace_bytes(e3.E3_CALL_MASKED_MEAN_ENTROPY, 131072) >= 16
+    assert e3.e3_workspace_bytes(e3.E3_CALL_MASKED_MEAN_ENTROPY, 0) >= 16
+
+
+def test_device_calls_reject_bad_arguments_on_the_host(e3):
+    L = e3.lib()
+    # checked before any CUDA call is made, so these run without a device
+    assert L.e3_sample(None, 7, 1, 8, 8, None, 0, 0, 0, 0, None, None, None, None, 0, None) == 2   # dtype
+    assert L.e3_sample(None, 0, -1, 8, 8, None, 0, 0, 0, 0, None, None, None, None, 0, None) == 1  # rows < 0
+    assert L.e3_sample(None, 0, 1, 8, 4, None, 0, 0, 0, 0, None, None, None, None, 0, None) == 1   # stride < V
+    assert L.e3_sample(None, 0, 1, 1 << 31, 1 << 31, None, 0, 0, 0, 0, None, None, None, None, 0, None) == 1
+    assert L.e3_sample(None, 0, 0, 8, 8, None, 0, 0, 0, 0, None, None, None, None, 0, None) == 0   # rows == 0
+    assert L.e3_sample(None, 0, 0, 8, 8, None, 0, 1 << 56, 0, 0, None, None, None, None, 0, None) == 1
+    assert L.e3_sample(None, 0, 0, 8, 8, None, 0, 0, 0, 2, None, None, None, None, 0, None) == 1   # sampler
+    assert L.e3_sample(1024, 0, 1, 8, 8, None, 0, 0, 0, 0, None, None, None, None, 0, None) == 1   # temps NULL
+    assert L.e3_sample(1026, 0, 1, 8, 8, 1024, 0, 0, 0, 0, 1024, None, None, None, 0, None) == 3   # misaligned
+    assert L.e3_token_logp_entropy(None, 0, 0, 8, 8, None, None, None, 1.0, None, None, None, 0, None) == 0
+    assert L.e3_token_logp_entropy(1024, 0, 1, 8, 8, None, None, None, 1.0, None, None, None, 0, None) == 1
+    assert L.e3_masked_mean_entropy(None, None, -1, None, None, None, 0, None) == 1
+    assert L.e3_masked_mean_entropy(1024, None, 4, 1024, 1032, None, 0, None) == 4                  # workspace
+    assert L.e3_group_advantage(None, None, 0, 1e-6, 1, None, None, None) == 0
+    assert L.e3_group_advantage(None, None, 2, 1e-6, 1, None, None, None) == 1
+    with pytest.raises(ValueError):
+        import torch
+        e3.e3_sample(torch.zeros(2, 8), torch.ones(2), 0, 0)   # CPU tensors: there is no CPU path
+
+
+def test_allocate_budget_matches_oracle(e3):
+    rng = np.random.default_rng(11)
+    for trial in range(400):
+        B = int(rng.integers(1, 80))
+        G = int(rng.integers(1, 20))
+        G_min = int(rng.integers(0, G + 1))
+        G_max = int(rng.integers(G, 2 * G + 6))
+        if trial % 4 == 0:
+            k = rng.integers(1, B + 1, size=B) / B     # normalised ranks, with ties
+        elif trial % 4 == 1:
+            k = np.round(rng.random(B), 1)
+        else:
+            k = rng.beta(2, 2, size=B)
+        for mode in (0, 1):
+            got = e3.e3_allocate_budget(k.tolist(), G, G_min, G_max, mode)
+            ref = oracle.allocate_budget(k, G, G_min, G_max, mode)
+            assert got == ref.tolist(), (B, G, G_min, G_max, mode)
+            assert sum(got) == B * G
+    assert e3.e3_allocate_budget([], 8, 4, 12) == []
+    assert e3.e3_allocate_budget([0.0, 0.0], 8, 4, 12) == [8, 8]
+    for args in (([0.5], 8, 9, 12), ([0.5], 8, 4, 7)):
+        with pytest.raises(e3.E3Error) as ei:
+            e3.e3_allocate_budget(*args)
+        assert ei.value.status == 5
+    for bad in ([1.5], [-0.1], [float("nan")]):
+        with pytest.raises(e3.E3Error) as ei:
+            e3.e3_allocate_budget(bad, 8, 4, 12)
+        assert ei.value.status == 1
+
+
+def test_update_temperature_matches_oracle(e3):
+    rng = np.random.default_rng(12)
+    for trial in range(200):
+        kw = dict(tau=float(rng.uniform(0.3, 2.0)), H_init=float(rng.uniform(0.05, 1.0)) if trial % 5 else float("nan"),
+                  t=int(rng.integers(0, 500)), t_anneal=288, t_max=480, eta=float(rng.uniform(0.5, 0.99)),
+                  V=int(rng.choice([32000, 151936, 256000])))
+        if trial % 7 == 0:
+            kw.update(tau_min=0.5, tau_max=1.5)
+        a, b = e3.make_sched(**kw), oracle.make_sched(**kw)
+        for _ in range(5):
+            H = float(rng.uniform(0.02, 1.5))
+            ta = e3.e3_update_temperature(a, H)
+            tb = oracle.update_temperature(b, H)
+            assert ta == pytest.approx(tb, rel=1e-12)
+            assert a.t == b.t and a.H_init == b.H_init
+            assert e3.e3_anneal_target(a) == pytest.approx(oracle.anneal_target(b), rel=1e-12)
+    s = e3.make_sched(tau=1.0, H_init=0.2)
+    for bad in (0.0, -1.0, float("nan"), float("inf")):
+        with pytest.raises(e3.E3Error):
+            e3.e3_update_temperature(s, bad)
+    assert s.tau == 1.0 and s.t == 0
+    # an update that would push tau below zero is refused and leaves the state alone
+    s = e3.make_sched(tau=4.0, H_init=1e-9, V=3)
+    with pytest.raises(e3.E3Error):
+        e3.e3_update_temperature(s, 1e3)
+    assert s.tau == 4.0 and s.t == 0
