@@ -1,0 +1,370 @@
+#!/usr/bin/env python
+"""Benchmark of the vocabulary-side hot path on B200.
+
+One "step" is one pass of the whole path over one synthetic rollout batch shaped like the
+paper's (64 prompts x 8 rollouts = 512 rows, V = 151,936, bf16 logits):
+
+    256 decode steps of e3_sample (fused temperature softmax + entropy + log-prob + Gumbel-max
+        sample; the logits rotate through a ring of 8 distinct buffers = 1.24 GB, larger than L2,
+        the Philox step counter advances every launch)
+  + one e3_token_logp_entropy over the ring's 4,096 rows (the training forward of those tokens)
+  + e3_masked_mean_entropy over their entropies
+  + e3_group_advantage over the 512 rollouts (64 groups of 8)
+  + the host temperature update fed by the mean entropy (16 bytes device -> host).
+
+`value` = logit rows per second over all ranks with the logits resident in HBM.  `e2e` = the
+same step with the logits in pinned HOST memory: every decode step copies its logits host ->
+device and its tokens device -> host inside the timed region.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--sampler 0|1] [--impl e3|reference]
+
+Under torchrun (N > 1) every rank runs the same per-GPU batch with its own row_base (weak
+scaling; rows are independent, the only exchange is a 16-byte all-reduce of the entropy sum
+and count).  `--impl reference` times the fp64 CPU oracle on a bounded sample of the same
+workload on the host cores (rank 0 only).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+ROWS, V, DECODE_STEPS, RING = 512, 151936, 256, 8
+GROUP = 8
+METRIC = "logit rows/s, fused sample+entropy, V=151,936"
+UNIT = "rows/s"
+WORKLOAD = "rollout decode step: 512 rows (64 prompts x 8 rollouts) x V=151,936 bf16, 256 decode steps"
+
+
+def _peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        try:
+            return float(json.load(open(path))["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.lines = index, None, []
+
+    def __enter__(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+        return self
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def __exit__(self, *a):
+        if self.proc is not None:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except Exception:
+                self.proc.kill()
+
+    def summary(self):
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.lines:
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) < 6:
+                continue
+            try:
+                sm.append(float(parts[0])); mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[2:6]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def cpu_baseline(sampler: int, budget_s: float = 12.0):
+    """The oracle as it stands, timed on the host cores on a bounded sample of the workload's rows."""
+    import torch
+    import oracle
+    from paper_2505_18573_b200 import inputs
+    oracle.build()
+    probe_rows = 16
+    logits = inputs.zipf_gaussian_logits(64, V, seed=10, dtype=torch.bfloat16)
+    temps = inputs.uniform_temps(64, seed=2).numpy()
+    arr = inputs.to_oracle_array(logits)
+    t0 = time.perf_counter()
+    oracle.sample(arr[:probe_rows], temps[:probe_rows], 0, 0, 0, sampler)
+    per_row = (time.perf_counter() - t0) / probe_rows
+    n = int(max(64, min(32768, budget_s / max(per_row, 1e-9))))
+    reps = (n + 63) // 64
+    t0 = time.perf_counter()
+    for r in range(reps):
+        oracle.sample(arr, temps, 0, r, 0, sampler)
+    dt = time.perf_counter() - t0
+    rows = reps * 64
+    return {"value": rows / dt, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": f"{rows} rows of the workload's logits (64 distinct rows x {reps} step counters), "
+                      f"sampler {sampler}, {dt:.1f} s"}
+
+
+def run_reference(args, rank: int):
+    """Reference arm = the CPU oracle (there is no other implementation of the paper's path)."""
+    if rank != 0:
+        return
+    import numpy as np
+    import torch
+    import oracle
+    from paper_2505_18573_b200 import inputs
+    oracle.build()
+    rows = 256
+    logits = inputs.to_oracle_array(inputs.zipf_gaussian_logits(rows, V, seed=10, dtype=torch.bfloat16))
+    temps = inputs.uniform_temps(rows, seed=2).numpy()
+    for w in range(args.warmup):
+        oracle.sample(logits[:16], temps[:16], 0, w, 0, args.sampler)
+    times = []
+    for k in range(args.steps):
+        t0 = time.perf_counter()
+        r = oracle.sample(logits, temps, 0, 1000 + k, 0, args.sampler)
+        oracle.token_logp_entropy(logits[:8], r.tok[:8], temp_scalar=1.0)
+        oracle.masked_mean_entropy(r.ent.astype(np.float32), None)
+        oracle.group_advantage((r.tok % 2).astype(np.float32), np.arange(0, rows + 1, GROUP))
+        times.append(time.perf_counter() - t0)
+    total = sum(times)
+    value = (rows + 8) * args.steps / total
+    sample = f"{rows} sampled rows + 8 training-side rows of the workload per step (full workload: 135,168 rows)"
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "sampler": args.sampler, "sample": sample},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+                             "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--sampler", type=int, default=0, choices=[0, 1])
+    ap.add_argument("--impl", default="e3", choices=["e3", "reference"])
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--profile-launches", type=int, default=0,
+                    help="run this many decode launches plus one training-side launch and exit (for ncu captures)")
+    args = ap.parse_args()
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2505_18573_b200 import binding as e3
+    from paper_2505_18573_b200 import inputs
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the path has no CPU fallback")
+    e3.lib()
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    # ---- synthetic batch, resident in HBM --------------------------------------------------------
+    row_base = rank * ROWS
+    batch = torch.empty((RING * ROWS, V), dtype=torch.bfloat16, device=dev)   # the ring, also the training batch
+    ring = [batch[i * ROWS:(i + 1) * ROWS] for i in range(RING)]
+    for i in range(RING):
+        ring[i].copy_(inputs.zipf_gaussian_logits(ROWS, V, seed=10 + i + 1000 * rank, dtype=torch.bfloat16, device=dev))
+    temps = inputs.uniform_temps(ROWS, seed=2 + 1000 * rank, device=dev)
+    all_toks = torch.zeros(RING * ROWS, dtype=torch.int32, device=dev)
+    toks = [all_toks[i * ROWS:(i + 1) * ROWS] for i in range(RING)]
+    sizes = [GROUP] * (ROWS // GROUP)
+    rewards = inputs.bernoulli_rewards(sizes, 0.5, seed=3 + rank, device=dev)
+    offsets = inputs.group_offsets(sizes, device=dev)
+    mask, _ = inputs.response_mask(RING, ROWS, seed=5 + rank, min_len=ROWS // 8, device=dev)
+    logp = torch.empty(ROWS, dtype=torch.float32, device=dev)
+    ent = torch.empty(ROWS, dtype=torch.float32, device=dev)
+    t_logp = torch.empty(RING * ROWS, dtype=torch.float32, device=dev)
+    t_ent = torch.empty(RING * ROWS, dtype=torch.float32, device=dev)
+    adv = torch.empty(ROWS, dtype=torch.float32, device=dev)
+    flags = torch.empty(ROWS // GROUP, dtype=torch.uint8, device=dev)
+    mean_out = torch.empty(2, dtype=torch.float64, device=dev)
+    ws = torch.empty(e3.e3_workspace_bytes(e3.E3_CALL_MASKED_MEAN_ENTROPY, RING * ROWS), dtype=torch.uint8, device=dev)
+    mean_host = torch.empty(2, dtype=torch.float64).pin_memory()
+    sched = e3.make_sched(tau=1.0, V=V, t_anneal=288, t_max=480, eta=0.9)
+    stream = torch.cuda.current_stream()
+    launches_per_step = DECODE_STEPS + 1 + 2 + 1
+
+    def decode_loop(step_index):
+        for d in range(DECODE_STEPS):
+            b = d % RING
+            e3.e3_sample(ring[b], temps, 0, step_index * DECODE_STEPS + d, row_base, args.sampler,
+                         out_tok=toks[b], out_logp=logp, out_ent=ent)
+
+    def tail(step_index):
+        e3.e3_token_logp_entropy(batch, all_toks, mask=mask, temp_scalar=float(sched.tau),
+                                 out_logp=t_logp, out_ent=t_ent)
+        e3.e3_masked_mean_entropy(t_ent, mask, out=mean_out, workspace=ws)
+        e3.e3_group_advantage(rewards, offsets, out_adv=adv, out_flags=flags)
+        if world > 1:
+            sc = mean_out.clone()
+            sc[0] = sc[0] * sc[1]
+            dist.all_reduce(sc)
+            sc[0] = sc[0] / sc[1]
+            mean_host.copy_(sc, non_blocking=True)
+        else:
+            mean_host.copy_(mean_out, non_blocking=True)
+        stream.synchronize()
+        e3.e3_update_temperature(sched, float(mean_host[0]))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    if args.profile_launches > 0:
+        for d in range(args.profile_launches):
+            e3.e3_sample(ring[d % RING], temps, 0, d, row_base, args.sampler, out_tok=toks[d % RING],
+                         out_logp=logp, out_ent=ent)
+        e3.e3_token_logp_entropy(batch, all_toks, mask=mask, temp_scalar=1.0, out_logp=t_logp, out_ent=t_ent)
+        torch.cuda.synchronize()
+        print(json.dumps({"profile_launches": args.profile_launches}), flush=True)
+        return
+
+    for w in range(args.warmup):
+        decode_loop(w); tail(w)
+
+    # ---- timed region: K steps, logits resident ----------------------------------------------------
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    dec_ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    tail_ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    barrier()
+    with ClockSampler(local_rank) as clocks:
+        ev0.record()
+        for k in range(args.steps):
+            dec_ev[k][0].record()
+            decode_loop(args.warmup + k)
+            dec_ev[k][1].record()
+            tail(args.warmup + k)
+            tail_ev[k].record()
+        ev1.record()
+        barrier()
+    ms_total = ev0.elapsed_time(ev1)
+    ms_decode = sum(a.elapsed_time(b) for a, b in dec_ev)
+    ms_tail = sum(dec_ev[k][1].elapsed_time(tail_ev[k]) for k in range(args.steps))
+    tmax = torch.tensor([ms_total], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+    ms_total_max = float(tmax[0])
+    rows_per_step = (DECODE_STEPS + RING) * ROWS
+    value = world * rows_per_step * args.steps / (ms_total_max * 1e-3)
+
+    # ---- end to end: logits in pinned host memory --------------------------------------------------
+    e2e = None
+    if args.e2e_steps > 0:
+        host_ring = [torch.empty((ROWS, V), dtype=torch.bfloat16).pin_memory() for _ in range(RING)]
+        for h, d in zip(host_ring, ring):
+            h.copy_(d)
+        stage = [torch.empty((ROWS, V), dtype=torch.bfloat16, device=dev) for _ in range(2)]
+        tok_host = torch.empty((DECODE_STEPS, ROWS), dtype=torch.int32).pin_memory()
+        temps_host = temps.cpu().pin_memory()
+        torch.cuda.synchronize()
+
+        def e2e_step(step_index):
+            tdev = temps_host.to(dev, non_blocking=True)
+            for d in range(DECODE_STEPS):
+                s = stage[d % 2]
+                s.copy_(host_ring[d % RING], non_blocking=True)
+                e3.e3_sample(s, tdev, 0, step_index * DECODE_STEPS + d, row_base, args.sampler,
+                             out_tok=toks[d % RING], out_logp=logp, out_ent=ent)
+                tok_host[d].copy_(toks[d % RING], non_blocking=True)
+            for b in range(RING):
+                sl = slice(b * ROWS, (b + 1) * ROWS)
+                s = stage[b % 2]
+                s.copy_(host_ring[b], non_blocking=True)
+                e3.e3_token_logp_entropy(s, toks[b], mask=mask[sl], temp_scalar=float(sched.tau),
+                                         out_logp=t_logp[sl], out_ent=t_ent[sl])
+            e3.e3_masked_mean_entropy(t_ent, mask, out=mean_out, workspace=ws)
+            e3.e3_group_advantage(rewards, offsets, out_adv=adv, out_flags=flags)
+            mean_host.copy_(mean_out, non_blocking=True)
+            stream.synchronize()
+            e3.e3_update_temperature(sched, float(mean_host[0]))
+
+        e2e_step(10_000)
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for k in range(args.e2e_steps):
+            e2e_step(10_001 + k)
+        e1.record()
+        barrier()
+        e2e_ms = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device=dev)
+        if world > 1:
+            dist.all_reduce(e2e_ms, op=dist.ReduceOp.MAX)
+        e2e = {"value": world * rows_per_step * args.e2e_steps / (float(e2e_ms[0]) * 1e-3), "unit": UNIT,
+               "h2d_bytes_per_step": (DECODE_STEPS + RING) * ROWS * V * 2 + ROWS * 4,
+               "d2h_bytes_per_step": DECODE_STEPS * ROWS * 4 + 16}
+
+    if rank == 0:
+        peak, peak_kind = _peaks()
+        bytes_per_launch = ROWS * V * 2 + ROWS * 4 + ROWS * 12
+        launch_s = ms_decode * 1e-3 / (args.steps * DECODE_STEPS)
+        achieved = bytes_per_launch / launch_s / 1e9
+        unmasked = int(mask.sum().item())
+        train_bytes = unmasked * V * 2
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_total_max / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "logits": "bf16", "sampler": args.sampler, "rows_per_gpu": ROWS, "V": V,
+                       "decode_steps": DECODE_STEPS, "l2": f"ring of {RING} logits buffers (1.24 GB) larger than L2",
+                       "step": "256 x e3_sample + e3_token_logp_entropy(4096 rows) + masked mean + group advantage + host tau update",
+                       "e2e_steps": args.e2e_steps},
+            "roofline": {"bound": "hbm", "kernel": "rows_kernel (e3_sample, bf16)", "achieved": achieved, "peak": peak,
+                         "peak_kind": peak_kind, "unit": "GB/s", "frac": achieved / peak, "frac_of_8TBs": achieved / 8000.0,
+                         "us_per_launch": launch_s * 1e6, "bytes_per_launch": bytes_per_launch, "traffic": None},
+            "training_side": {"ms_per_step": ms_tail / args.steps, "unmasked_rows": unmasked,
+                              "GBps_incl_small_kernels_and_sync": train_bytes / (ms_tail * 1e-3 / args.steps) / 1e9},
+            "e2e": e2e,
+            "gpu_launches": launches_per_step * args.steps,
+            "clocks": clocks.summary(),
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            line["cpu_baseline"] = cpu_baseline(args.sampler)
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
