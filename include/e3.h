@@ -138,6 +138,34 @@ E3_API e3_status e3_masked_mean_entropy(const float *ent, const uint8_t *mask, i
                                  void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * The same mean entropy for callers that have no scratch memory to give.  (The paper has no
+ * counterpart for this entry point; it exists for deployment reasons only.)
+ *
+ * Who needs it: code that runs where device allocation is off limits -- a plugin or callback
+ * executing inside somebody else's stream or inference engine, a real-time loop that must not
+ * touch the allocator, a process whose memory pool was sized up front and handed out completely.
+ * Such callers cannot call cudaMalloc and often have no spare buffer for
+ * e3_masked_mean_entropy's workspace.  Here the per-block partial sums live in a fixed
+ * 16 KiB array inside the library image; every GPU that loads the library holds those 16 KiB
+ * until the process exits.  The call itself allocates and frees nothing.
+ *
+ *   ent, mask, n, out_mean, out_count, stream: as in e3_masked_mean_entropy (device pointers).
+ *   n may not exceed E3_STATIC_MEAN_MAX_TOKENS; a larger n returns E3_ERR_WORKSPACE (the
+ *   built-in scratch is not sized for it) and launches nothing.
+ *
+ * The first call on each device looks up the array's device address (one runtime query, made
+ * with that device current).  Make that first call outside any stream capture.
+ * All calls on a device share the one array, and it keeps whatever the previous call left in it.
+ * That is harmless for calls that run one after another (each call overwrites every entry it
+ * later reads), but two calls whose kernels overlap on the GPU -- different streams, no
+ * ordering between them -- race on it and give wrong means.  Serialise them.
+ * Results equal e3_masked_mean_entropy's bit for bit.
+ */
+#define E3_STATIC_MEAN_MAX_TOKENS (INT64_C(1) << 26)
+E3_API e3_status e3_masked_mean_entropy_static(const float *ent, const uint8_t *mask, int64_t n,
+                                               double *out_mean, double *out_count, void *stream);
+
+/*
  * Group-relative advantage (Eq. "adv"): inside each rollout group g = rows
  * [group_offsets[g], group_offsets[g+1]):  A_i = (r_i - mean) / (std + eps).
  * Groups may have any size (the rollout budget of Algorithm 1 makes them ragged).

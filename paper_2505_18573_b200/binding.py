@@ -22,7 +22,7 @@ E3_CALL_SAMPLE, E3_CALL_TOKEN_LOGP_ENTROPY, E3_CALL_MASKED_MEAN_ENTROPY = 0, 1, 
 E3_SAMPLE_BLOCK = 256
 
 EXPORTS = ("e3_status_string", "e3_workspace_bytes", "e3_sample", "e3_token_logp_entropy",
-           "e3_masked_mean_entropy", "e3_group_advantage", "e3_allocate_budget", "e3_update_temperature",
+           "e3_masked_mean_entropy", "e3_masked_mean_entropy_static", "e3_group_advantage", "e3_allocate_budget", "e3_update_temperature",
            "e3_anneal_target")
 
 
@@ -64,6 +64,9 @@ def lib() -> C.CDLL:
         L.e3_masked_mean_entropy.restype = C.c_int
         L.e3_masked_mean_entropy.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p,
                                              C.c_size_t, C.c_void_p]
+        L.e3_masked_mean_entropy_static.restype = C.c_int
+        L.e3_masked_mean_entropy_static.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p,
+                                                    C.c_void_p]
         L.e3_group_advantage.restype = C.c_int
         L.e3_group_advantage.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_float, C.c_int, C.c_void_p,
                                          C.c_void_p, C.c_void_p]
@@ -181,6 +184,30 @@ def e3_masked_mean_entropy(ent, mask=None, out=None, workspace=None, stream=None
     st = lib().e3_masked_mean_entropy(_ptr(ent), _ptr(mask), n, out.data_ptr(), out.data_ptr() + 8,
                                       _ptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream))
     _check("e3_masked_mean_entropy", st)
+    return out
+
+
+E3_STATIC_MEAN_MAX_TOKENS = 1 << 26
+
+
+def e3_masked_mean_entropy_static(ent, mask=None, out=None, stream=None):
+    """Mean entropy without any scratch buffer from the caller (for code that may not allocate
+    device memory: plugins inside another engine's stream, fixed-pool or real-time processes).
+    The partial sums use a 16 KiB array built into the library, shared by every call on the
+    device, so calls must not overlap on the GPU.  ``out`` (float64 CUDA tensor [2] = mean, count)
+    must be passed by callers that really cannot allocate; when omitted it is created here with
+    torch for convenience.  Raises E3Error(E3_ERR_WORKSPACE) above E3_STATIC_MEAN_MAX_TOKENS."""
+    _dev(ent, "ent"); _dev(mask, "mask")
+    if ent.dtype != torch.float32 or not ent.is_contiguous():
+        raise ValueError("ent must be a contiguous float32 tensor")
+    n = ent.numel()
+    if mask is not None and (mask.dtype != torch.uint8 or mask.numel() != n):
+        raise ValueError("mask must be uint8 with one entry per token")
+    if out is None:
+        out = torch.empty(2, dtype=torch.float64, device=ent.device)
+    st = lib().e3_masked_mean_entropy_static(_ptr(ent), _ptr(mask), n, out.data_ptr(), out.data_ptr() + 8,
+                                             _stream(stream))
+    _check("e3_masked_mean_entropy_static", st)
     return out
 
 
