@@ -70,9 +70,10 @@ typedef enum {
 /* Human-readable name of a status code (static string). */
 E3_API const char *e3_status_string(e3_status s);
 
-/* Bytes of device scratch a call needs for the given problem size (0 = none;
- * the call then accepts workspace == NULL).  For E3_CALL_MASKED_MEAN_ENTROPY
- * `rows` is the number of tokens n and V, dt are ignored. */
+/* Bytes of device scratch a call uses for the given problem size.  For
+ * E3_CALL_MASKED_MEAN_ENTROPY `rows` is the number of tokens n and V, dt are ignored.
+ * Scratch contents on entry never matter.  A workspace must not be shared by calls that can run
+ * at the same time (different streams without ordering).  It must be 16-byte aligned. */
 E3_API size_t e3_workspace_bytes(e3_call which, int64_t rows, int64_t V, e3_dtype dt);
 
 /*
@@ -97,7 +98,10 @@ E3_API size_t e3_workspace_bytes(e3_call which, int64_t rows, int64_t V, e3_dtyp
  *               Sampler 1: u_b = (x_b + 1/2) 2^-32, x_b word (b mod 4) of call b/4 of stream 2, for block b;
  *               the in-block draw uses word 0 of call 0 of stream 3.
  *   out_tok     device int32 [rows], required.   out_logp, out_ent: device float [rows], each may be NULL.
- *   workspace   device scratch of e3_workspace_bytes(E3_CALL_SAMPLE, ...) bytes (NULL when that is 0).
+ *   workspace   device scratch of e3_workspace_bytes(E3_CALL_SAMPLE, ...) bytes.  It holds the partial states
+ *               of rows that are split between thread blocks so that every block streams the same number
+ *               of bytes.  NULL (or too small) is accepted: rows are then never split, which costs
+ *               throughput when there are fewer than a few thousand rows.
  * -inf logits are allowed (probability 0, never drawn).
  */
 E3_API e3_status e3_sample(const void *logits, e3_dtype dt, int64_t rows, int64_t V, int64_t row_stride,

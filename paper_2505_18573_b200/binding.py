@@ -125,9 +125,24 @@ def e3_workspace_bytes(which: int, rows: int, V: int = 0, dt: int = E3_F32) -> i
     return int(lib().e3_workspace_bytes(which, rows, V, dt))
 
 
+_row_workspaces = {}
+
+
+def _row_workspace(device, stream_handle: int, which: int, rows: int, V: int, dt: int):
+    """Scratch for the row kernels, one buffer per (device, stream): calls that may overlap on the GPU
+    must not share a workspace.  Callers that manage memory themselves pass ``workspace=`` instead."""
+    key = (device.index, stream_handle)
+    need = e3_workspace_bytes(which, rows, V, dt)
+    ws = _row_workspaces.get(key)
+    if ws is None or ws.numel() < need:
+        ws = torch.empty(max(need, 16), dtype=torch.uint8, device=device)
+        _row_workspaces[key] = ws
+    return ws
+
+
 def e3_sample(logits, temps, seed: int, counter: int, row_base: int = 0, sampler: int = E3_SAMPLER_TOKEN,
               out_tok=None, out_logp=None, out_ent=None, want_logp: bool = True, want_ent: bool = True,
-              stream=None):
+              workspace=None, stream=None):
     """Rollout step: returns (tok int32, logp float32 | None, ent float32 | None), each [rows]."""
     dt, rows, V, stride = _logits_desc(logits)
     _dev(temps, "temps")
@@ -140,14 +155,18 @@ def e3_sample(logits, temps, seed: int, counter: int, row_base: int = 0, sampler
         out_logp = torch.empty(rows, dtype=torch.float32, device=dev)
     if out_ent is None and want_ent:
         out_ent = torch.empty(rows, dtype=torch.float32, device=dev)
+    sh = _stream(stream)
+    if workspace is None:
+        workspace = _row_workspace(dev, sh, E3_CALL_SAMPLE, rows, V, dt)
     st = lib().e3_sample(_ptr(logits), dt, rows, V, stride, _ptr(temps), seed, counter, row_base, sampler,
-                         _ptr(out_tok), _ptr(out_logp), _ptr(out_ent), None, 0, _stream(stream))
+                         _ptr(out_tok), _ptr(out_logp), _ptr(out_ent), _ptr(workspace),
+                         workspace.numel() * workspace.element_size(), sh)
     _check("e3_sample", st)
     return out_tok, out_logp, out_ent
 
 
 def e3_token_logp_entropy(logits, targets, mask=None, temps=None, temp_scalar: float = 1.0, out_logp=None,
-                          out_ent=None, stream=None):
+                          out_ent=None, workspace=None, stream=None):
     """Training-side pass: returns (logp float32, ent float32), each [rows]; masked rows give 0."""
     dt, rows, V, stride = _logits_desc(logits)
     _dev(targets, "targets"); _dev(mask, "mask"); _dev(temps, "temps")
@@ -162,8 +181,12 @@ def e3_token_logp_entropy(logits, targets, mask=None, temps=None, temp_scalar: f
         out_logp = torch.empty(rows, dtype=torch.float32, device=dev)
     if out_ent is None:
         out_ent = torch.empty(rows, dtype=torch.float32, device=dev)
+    sh = _stream(stream)
+    if workspace is None:
+        workspace = _row_workspace(dev, sh, E3_CALL_TOKEN_LOGP_ENTROPY, rows, V, dt)
     st = lib().e3_token_logp_entropy(_ptr(logits), dt, rows, V, stride, _ptr(targets), _ptr(mask), _ptr(temps),
-                                     float(temp_scalar), _ptr(out_logp), _ptr(out_ent), None, 0, _stream(stream))
+                                     float(temp_scalar), _ptr(out_logp), _ptr(out_ent), _ptr(workspace),
+                                     workspace.numel() * workspace.element_size(), sh)
     _check("e3_token_logp_entropy", st)
     return out_logp, out_ent
 

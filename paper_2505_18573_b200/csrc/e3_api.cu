@@ -39,8 +39,8 @@ extern "C" size_t e3_workspace_bytes(e3_call which, int64_t rows, int64_t V, e3_
   (void)V;
   (void)dt;
   switch (which) {
-    case E3_CALL_SAMPLE: return 0;
-    case E3_CALL_TOKEN_LOGP_ENTROPY: return 0;
+    case E3_CALL_SAMPLE: return e3::rows_workspace_bytes();
+    case E3_CALL_TOKEN_LOGP_ENTROPY: return e3::rows_workspace_bytes();
     case E3_CALL_MASKED_MEAN_ENTROPY: return e3::mean_workspace_bytes(rows < 0 ? 0 : rows);
   }
   return 0;
@@ -50,10 +50,9 @@ extern "C" e3_status e3_sample(const void *logits, e3_dtype dt, int64_t rows, in
                                const float *temps, uint64_t seed, uint64_t counter, int64_t row_base,
                                e3_sampler sampler, int32_t *out_tok, float *out_logp, float *out_ent,
                                void *workspace, size_t workspace_bytes, void *stream) {
-  (void)workspace;
-  (void)workspace_bytes;
   e3_status st = check_logits(logits, dt, rows, V, row_stride);
   if (st != E3_OK) return st;
+  if (misaligned(workspace, 16)) return E3_ERR_ALIGNMENT;
   if (sampler != E3_SAMPLER_TOKEN && sampler != E3_SAMPLER_BLOCK) return E3_ERR_INVALID_ARG;
   if (row_base < 0 || counter >= (uint64_t(1) << 56)) return E3_ERR_INVALID_ARG;
   if (rows == 0) return E3_OK;
@@ -71,7 +70,8 @@ extern "C" e3_status e3_sample(const void *logits, e3_dtype dt, int64_t rows, in
   p.row_base = static_cast<uint32_t>(row_base);
   p.mode = e3::kModeSample;
   cudaError_t e = e3::launch_rows(p, static_cast<int>(dt), static_cast<int>(sampler),
-                                  rows_are_16B_aligned(logits, dt, row_stride), static_cast<cudaStream_t>(stream));
+                                  rows_are_16B_aligned(logits, dt, row_stride), workspace, workspace_bytes,
+                                  static_cast<cudaStream_t>(stream));
   return e == cudaSuccess ? E3_OK : E3_ERR_CUDA;
 }
 
@@ -79,10 +79,9 @@ extern "C" e3_status e3_token_logp_entropy(const void *logits, e3_dtype dt, int6
                                            int64_t row_stride, const int32_t *targets, const uint8_t *mask,
                                            const float *temps, float temp_scalar, float *out_logp, float *out_ent,
                                            void *workspace, size_t workspace_bytes, void *stream) {
-  (void)workspace;
-  (void)workspace_bytes;
   e3_status st = check_logits(logits, dt, rows, V, row_stride);
   if (st != E3_OK) return st;
+  if (misaligned(workspace, 16)) return E3_ERR_ALIGNMENT;
   if (rows == 0) return E3_OK;
   if (!targets) return E3_ERR_INVALID_ARG;
   if (misaligned(targets, 4) || misaligned(temps, 4) || misaligned(out_logp, 4) || misaligned(out_ent, 4))
@@ -95,7 +94,7 @@ extern "C" e3_status e3_token_logp_entropy(const void *logits, e3_dtype dt, int6
   p.out_logp = out_logp; p.out_ent = out_ent;
   p.mode = e3::kModeTargets;
   cudaError_t e = e3::launch_rows(p, static_cast<int>(dt), -1, rows_are_16B_aligned(logits, dt, row_stride),
-                                  static_cast<cudaStream_t>(stream));
+                                  workspace, workspace_bytes, static_cast<cudaStream_t>(stream));
   return e == cudaSuccess ? E3_OK : E3_ERR_CUDA;
 }
 

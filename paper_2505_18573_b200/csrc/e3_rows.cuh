@@ -1,16 +1,20 @@
-// Shared declarations of the row-streaming kernels (host side of the launch and device parameters).
+// Shared declarations of the row-streaming kernel (host side of the launch and device parameters).
 #pragma once
 #include <cuda_runtime.h>
+#include <stddef.h>
 #include <stdint.h>
 
 namespace e3 {
 
-constexpr int kStreamWarps = 8;                     // warps that stream logits
+constexpr int kStreamWarps = 8;                     // warps that consume logits
 constexpr int kStreamThreads = kStreamWarps * 32;   // 256
-constexpr int kThreads = kStreamThreads + 32;       // + one warp that finishes rows
+constexpr int kThreads = kStreamThreads + 64;       // + one warp that issues bulk copies + one that finishes rows
 constexpr int kGroup = 16;                          // vocabulary entries per coarse Philox call
-constexpr int kSliceAlign = 512;                    // a CTA's slice of a row starts on a multiple of this
-constexpr int kMaxCluster = 8;
+constexpr int kTile = 512;                          // unit of the work split (entries); CTA ranges start on tile bounds
+constexpr int kChunk = 4096;                        // entries per pipeline stage (one 16-entry group per consumer thread)
+constexpr int kStages = 6;
+constexpr int kMaxGrid = 1024;                      // CTAs the piece workspace is sized for
+constexpr size_t kPieceBytes = 64;                  // one partial row state in the workspace
 
 enum RowsMode : int { kModeSample = 0, kModeTargets = 1 };
 
@@ -28,11 +32,22 @@ struct RowsParams {
   uint32_t ctr_lo;          // low word of the step counter
   uint32_t ctr_hi8;         // (high bits of the step counter) << 8; the stream tag is OR-ed in
   uint32_t row_base;
-  int64_t seg;              // vocabulary entries per CTA of a cluster (multiple of kSliceAlign)
   int mode;
+  // work split
+  int interleaved;          // 1: CTA b takes whole rows b, b + grid, ...; 0: contiguous tile ranges (rows may be cut)
+  int64_t tiles_per_row;    // ceil(V / kTile)
+  int64_t tiles_q, tiles_r; // total tiles = grid * tiles_q + tiles_r: CTA b starts at tile b*tiles_q + min(b, tiles_r)
+  // cut rows: pieces and arrival words in the caller's workspace
+  unsigned char *ws_pieces;          // [grid][2] pieces of kPieceBytes
+  unsigned long long *ws_arrivals;   // [grid] (call id << 16 | pieces arrived), for the row whose first tile CTA k holds
+  unsigned long long call_id;        // unique per call within the process (48 bits)
 };
 
-// Launches the streaming kernel for the given element type / sampler.  sampler: -1 = none (targets given).
-cudaError_t launch_rows(const RowsParams &p, int dtype, int sampler, bool aligned, cudaStream_t stream);
+size_t rows_workspace_bytes();
+
+// Launches the streaming kernel.  sampler: -1 = none (targets given), 0 = per-token Gumbel-max.
+// workspace may be nullptr: rows are then never cut (whole rows per CTA).
+cudaError_t launch_rows(RowsParams p, int dtype, int sampler, bool aligned, void *workspace, size_t workspace_bytes,
+                        cudaStream_t stream);
 
 }  // namespace e3

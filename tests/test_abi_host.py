@@ -34,7 +34,7 @@ def test_library_exports_every_declared_symbol(e3):
 def test_status_strings_and_workspace(e3):
     assert e3.status_string(0) == "E3_OK"
     assert e3.status_string(5) == "E3_ERR_INFEASIBLE"
-    assert e3.e3_workspace_bytes(e3.E3_CALL_SAMPLE, 512, 151936, e3.E3_BF16) == 0
+    assert e3.e3_workspace_bytes(e3.E3_CALL_SAMPLE, 512, 151936, e3.E3_BF16) >= 1024 * 136
     assert e3.e3_workspace_bytes(e3.E3_CALL_MASKED_MEAN_ENTROPY, 131072) >= 16
     assert e3.e3_workspace_bytes(e3.E3_CALL_MASKED_MEAN_ENTROPY, 0) >= 16
 
