@@ -12,8 +12,8 @@
 // waits for anybody.  (With a response mask, and when no workspace is given, CTAs take whole
 // rows round-robin instead.)
 //
-// Inside a CTA: one warp issues bulk asynchronous copies (cp.async.bulk, no multicast) of 4,096
-// entries into a 6-stage shared-memory ring guarded by mbarriers; eight warps consume the ring,
+// Inside a CTA: one warp issues bulk asynchronous copies (cp.async.bulk, no multicast) of 16 KiB
+// into a 6-stage shared-memory ring guarded by mbarriers; eight warps consume the ring,
 // each thread one 16-entry group per stage (= one coarse Philox call); one warp finishes rows
 // (merges the eight warp states, fp64 epilogue, piece protocol) so that the consumers never
 // stall on it.  Every mbarrier wait is bounded: when a wait runs out the CTA stops waiting
@@ -42,10 +42,10 @@
 namespace e3 {
 namespace {
 
-constexpr int kQueueCap = 160;
+constexpr int kQueueCap = 96;
 constexpr int kDrainAt = 32;
 constexpr int kSlots = 4;  // hand-over slots between the consumer warps and the finishing warp
-constexpr uint32_t kSpinLimit = 1u << 21;
+constexpr uint32_t kSpinLimit = 1u << 23;  // polls before a wait gives up (seconds)
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2f = 0.6931471805599453f;
 constexpr double kLn2 = 0.6931471805599453094;
@@ -79,7 +79,6 @@ struct Smem {
   unsigned long long best64;                         // (segment number << 32 | encoded best score) of sampler 0
   WarpPartial wpart[kSlots][kStreamWarps];
   int queue[kStreamWarps][kQueueCap];
-  int qcount[kStreamWarps];
   int timeout;                                       // set when a bounded wait ran out
 };
 
@@ -140,6 +139,7 @@ __device__ __forceinline__ void mbar_arrive(unsigned long long *b) {
 __device__ __forceinline__ void mbar_arrive_expect_tx(unsigned long long *b, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(b)), "r"(bytes) : "memory");
 }
+// One poll (the hardware may park the thread for a short, implementation-defined time).
 __device__ __forceinline__ bool mbar_try_wait(unsigned long long *b, uint32_t parity) {
   uint32_t ok;
   asm volatile(
@@ -150,14 +150,22 @@ __device__ __forceinline__ bool mbar_try_wait(unsigned long long *b, uint32_t pa
   return ok != 0;
 }
 // Bounded wait.  After any wait of the CTA has run out, no wait blocks any more.
-__device__ __forceinline__ void mbar_wait(unsigned long long *b, uint32_t parity, Smem &sm) {
-  if (mbar_try_wait(b, parity)) return;
+// sleep_ns > 0 parks the thread between polls (roles that mostly wait must not eat issue slots).
+__device__ __noinline__ void mbar_wait_slow(unsigned long long *b, uint32_t parity, Smem &sm, unsigned sleep_ns) {
   for (uint32_t it = 0; it < kSpinLimit; ++it) {
-    if (*reinterpret_cast<volatile int *>(&sm.timeout)) return;
     if (mbar_try_wait(b, parity)) return;
-    if (it > 32) __nanosleep(it > 4096 ? 256 : 32);
+    if (*reinterpret_cast<volatile int *>(&sm.timeout)) return;
+    if (sleep_ns) __nanosleep(sleep_ns);
   }
   *reinterpret_cast<volatile int *>(&sm.timeout) = 1;
+}
+__device__ __forceinline__ void mbar_wait(unsigned long long *b, uint32_t parity, Smem &sm, unsigned sleep_ns = 0) {
+  if (!mbar_try_wait(b, parity)) mbar_wait_slow(b, parity, sm, sleep_ns);
+}
+// Whole-warp wait with a single polling lane (used by the finishing warp, which mostly waits).
+__device__ __forceinline__ void mbar_wait_warp(unsigned long long *b, uint32_t parity, Smem &sm, int lane) {
+  if (lane == 0) mbar_wait(b, parity, sm, 512u);
+  __syncwarp();
 }
 __device__ __forceinline__ void bulk_copy_g2s(void *dst, const void *src, uint32_t bytes, unsigned long long *bar) {
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
@@ -229,24 +237,36 @@ __device__ __forceinline__ float load_group_guarded(const char *row, int64_t e0,
   return gmax;
 }
 
-// One full group from a pipeline stage in shared memory.  Returns the group's largest logit.
+// One full group: raw 16-byte words from a pipeline stage, then widening to fp32.
 template <int DT>
-__device__ __forceinline__ float load_group_smem(const unsigned char *stage, int tid, float (&z)[16]) {
+struct RawGroup {
+  uint4 q[DT == 0 ? 4 : 2];
+};
+
+template <int DT>
+__device__ __forceinline__ void load_raw_smem(const unsigned char *stage, int slot, RawGroup<DT> &r) {
+  constexpr int kQ = DT == 0 ? 4 : 2;
+  const uint4 *p = reinterpret_cast<const uint4 *>(stage) + slot * kQ;
+#pragma unroll
+  for (int i = 0; i < kQ; ++i) r.q[i] = p[i];
+}
+
+// Returns the group's largest logit.
+template <int DT>
+__device__ __forceinline__ float unpack_group(const RawGroup<DT> &r, float (&z)[16]) {
   if (DT == 0) {
-    const float4 *p = reinterpret_cast<const float4 *>(stage) + tid * 4;
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
-      const float4 v = p[q];
-      z[4 * q + 0] = v.x; z[4 * q + 1] = v.y; z[4 * q + 2] = v.z; z[4 * q + 3] = v.w;
+      z[4 * q + 0] = __uint_as_float(r.q[q].x); z[4 * q + 1] = __uint_as_float(r.q[q].y);
+      z[4 * q + 2] = __uint_as_float(r.q[q].z); z[4 * q + 3] = __uint_as_float(r.q[q].w);
     }
     float m[4];
 #pragma unroll
     for (int q = 0; q < 4; ++q) m[q] = fmaxf(fmaxf(z[4 * q], z[4 * q + 1]), fmaxf(z[4 * q + 2], z[4 * q + 3]));
     return fmaxf(fmaxf(m[0], m[1]), fmaxf(m[2], m[3]));
   } else {
-    const uint4 *p = reinterpret_cast<const uint4 *>(stage) + tid * 2;
-    const uint4 a = p[0], b = p[1];
-    const uint32_t w[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+    const uint32_t w[8] = {r.q[0].x, r.q[0].y, r.q[0].z, r.q[0].w, r.q[DT == 0 ? 0 : 1].x, r.q[DT == 0 ? 0 : 1].y,
+                           r.q[DT == 0 ? 0 : 1].z, r.q[DT == 0 ? 0 : 1].w};
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
       z[2 * j + 0] = __uint_as_float(w[j] << 16);
@@ -263,15 +283,21 @@ __device__ __forceinline__ float load_group_smem(const unsigned char *stage, int
 // CAREFUL also accepts -inf entries (skipped) and flags NaN; the fast form leaves NaN in the
 // sums when it meets either, which sends the thread's groups through the careful form once more.
 // ---------------------------------------------------------------------------------------------
+// The reference moves to max(R, gmax) before every group.  The fast form does this without a branch
+// (a per-lane branch that is rarely taken is taken by some lane of the warp almost every time):
+// the sums are multiplied by f = 2^(nRc_new - nRc_old), which is 1 when the reference stays.
+// Acc starts with nRc = kNoRef, a huge finite value, so that the first f is 0 and no inf*0 arises.
+constexpr float kNoRef = 1e30f;
+
 template <bool CAREFUL>
 __device__ __forceinline__ void accumulate(Acc &a, const float (&z)[16], float c, float gmax, int &err) {
-  if (gmax > a.R) {
-    if (gmax == CUDART_INF_F) {
-      err |= kErrValue;
-      return;
-    }
-    const float nRc = -gmax * c;
-    if (a.R != -CUDART_INF_F) {
+  if (CAREFUL) {
+    if (gmax > a.R) {
+      if (gmax == CUDART_INF_F) {
+        err |= kErrValue;
+        return;
+      }
+      const float nRc = -gmax * c;
       const float d = nRc - a.nRc;
       const float f = ex2f(d);
       if (f == 0.f) {
@@ -282,8 +308,19 @@ __device__ __forceinline__ void accumulate(Acc &a, const float (&z)[16], float c
         a.Z0 *= f;
         a.Z1 *= f;
       }
+      a.R = gmax;
+      a.nRc = nRc;
     }
-    a.R = gmax;
+  } else {
+    const float R = fmaxf(a.R, gmax);  // +inf or NaN logits end up as NaN in the sums and are sorted out later
+    const float nRc = -R * c;
+    const float d = nRc - a.nRc;       // <= 0
+    const float f = ex2f(d);
+    a.W0 = f * fmaf(d, a.Z0, a.W0);
+    a.W1 = f * fmaf(d, a.Z1, a.W1);
+    a.Z0 *= f;
+    a.Z1 *= f;
+    a.R = R;
     a.nRc = nRc;
   }
 #pragma unroll
@@ -329,18 +366,15 @@ struct EvalCtx {
   const char *row;
   float tau;
   uint32_t grow, ctr_lo, ctr_hi8, seg;
+  int V;
 };
 
-template <int DT>
-__device__ __noinline__ void eval_candidate(const EvalCtx &x, int i, Best &b, Smem &sm) {
-  const float zf = load_elem<DT>(x.row, i);
+// One entry with logit zf and coarse byte cbyte: screen with an fp32 upper bound, then evaluate in fp64.
+__device__ __noinline__ void eval_element(const EvalCtx &x, int i, uint32_t cbyte, float zf, Best &b, Smem &sm) {
   if (!(zf > b.zthr2) || zf == CUDART_INF_F) return;  // cannot win even with the largest Gumbel (also NaN, -inf)
-  const uint4 cw = philox(x.rk, (uint32_t)i >> 4, x.grow, x.ctr_lo, x.ctr_hi8 | 0u);
-  const uint32_t cbyte = (pick_word(cw, (i & 15) >> 2) >> (8 * (i & 3))) & 0xFFu;
   if (cbyte != 255u && !(zf > b.zthr)) return;
   const uint4 fw = philox(x.rk, (uint32_t)i >> 2, x.grow, x.ctr_lo, x.ctr_hi8 | 1u);
   const uint32_t xw = pick_word(fw, i & 3);
-  // fp32 upper bound of the score: skip the fp64 evaluation when even that cannot reach the best known score
   {
     float gh;
     if (cbyte == 255u) {
@@ -370,80 +404,204 @@ __device__ __noinline__ void eval_candidate(const EvalCtx &x, int i, Best &b, Sm
   }
 }
 
+// A queue entry names one 16-entry group: (group index << 5) | flags.  Flag bits 0-3: the coarse
+// bytes of word 0-3 contain 0xFF (may over-report); bit 4: some logit of the group is above the gate.
+// Each warp owns a queue; its fill count lives in a warp-uniform register, positions come from a
+// ballot, so queueing costs no atomics.  A chunk adds at most 32 entries per group slot, and the
+// queue is drained as soon as it holds 32, so kQueueCap >= 31 + 32 * (groups per thread) suffices.
 template <int DT>
-__device__ __forceinline__ void push_candidate(const EvalCtx &x, int i, Best &b, Smem &sm, int warp) {
-  const int slot = atomicAdd(&sm.qcount[warp], 1);
-  if (slot < kQueueCap)
-    sm.queue[warp][slot] = i;
-  else
-    eval_candidate<DT>(x, i, b, sm);
-}
-
-template <int DT>
-__device__ __forceinline__ void drain_queue(const EvalCtx &x, Best &b, Smem &sm, int warp, int lane, int at_least) {
-  __syncwarp();
-  int n = *reinterpret_cast<volatile int *>(&sm.qcount[warp]);
-  if (n < at_least) return;
-  n = n < kQueueCap ? n : kQueueCap;
-  for (int e = lane; e < n; e += 32) eval_candidate<DT>(x, sm.queue[warp][e], b, sm);
-  __syncwarp();
-  if (lane == 0) sm.qcount[warp] = 0;
-  __syncwarp();
-}
-
-// Gate, seed and queue for one group (sampler 0).  `seed` is warp-uniform: true on the warp's first
-// step of a segment, when nothing is known about the row's best score yet.
-template <int DT>
-__device__ __forceinline__ void sample_group(const EvalCtx &x, const float (&z)[16], float gmax, bool have, int e0,
-                                             int valid, Best &b, Smem &sm, int warp, bool seed) {
-  uint4 cb = make_uint4(0, 0, 0, 0);
-  if (have) cb = philox(x.rk, (uint32_t)e0 >> 4, x.grow, x.ctr_lo, x.ctr_hi8 | 0u);
-  if (seed) {
-    // A valid lower bound of the row's best score, from the coarse byte of the group's largest entry alone:
-    // u >= (c + 2^-33)/256  =>  g >= -ln(ln 256 - ln(c + 2^-33)).
-    float ylo = -CUDART_INF_F;
-    if (have && gmax > -CUDART_INF_F && gmax < CUDART_INF_F) {
-      uint32_t cbyte = 0;
+__device__ __noinline__ void eval_entry(const EvalCtx &x, int entry, Best &b, Smem &sm, bool aligned) {
+  const int base = (entry >> 5) << 4;
+  // all 16 logits of the group first (independent loads, one memory latency), then the coarse bytes
+  float z[16];
+  if (aligned && base + 16 <= x.V) {
+    if (DT == 0) {
+      const float4 *p = reinterpret_cast<const float4 *>(x.row) + (base >> 2);
 #pragma unroll
-      for (int k = 15; k >= 0; --k)
-        if (z[k] == gmax) cbyte = (pick_word(cb, k >> 2) >> (8 * (k & 3))) & 0xFFu;
-      const float neg_ln_u = (8.0f - lg2f((float)cbyte + 0x1p-33f)) * kLn2f;
-      const float glo = -lg2f(neg_ln_u) * kLn2f;
-      const float sf = gmax / x.tau;
-      ylo = sf - fabsf(sf) * 2e-6f + glo - 2e-3f;
+      for (int q = 0; q < 4; ++q) {
+        const float4 v = __ldg(p + q);
+        z[4 * q] = v.x; z[4 * q + 1] = v.y; z[4 * q + 2] = v.z; z[4 * q + 3] = v.w;
+      }
+    } else {
+      const uint4 *p = reinterpret_cast<const uint4 *>(x.row) + (base >> 3);
+#pragma unroll
+      for (int q = 0; q < 2; ++q) {
+        const uint4 v = __ldg(p + q);
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          z[8 * q + 2 * j] = __uint_as_float(w[j] << 16);
+          z[8 * q + 2 * j + 1] = __uint_as_float(w[j] & 0xFFFF0000u);
+        }
+      }
     }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) ylo = fmaxf(ylo, __shfl_xor_sync(0xffffffffu, ylo, o));
-    int enc = enc_float(ylo);
-    if ((threadIdx.x & 31) == 0 && enc > enc_neg_inf()) post_best(sm, x.seg, enc);
-    const int cta = read_best(sm, x.seg);
-    enc = enc > cta ? enc : cta;
-    if (enc > b.enc) set_gate(b, enc, x.tau);
   } else {
-    const int enc = read_best(sm, x.seg);
-    if (enc > b.enc) set_gate(b, enc, x.tau);
+    load_group_guarded<DT>(x.row, base, x.V - base, z);
   }
-  if (!have) return;
-  const uint32_t h = any_ff(cb.x) | any_ff(cb.y) | any_ff(cb.z) | any_ff(cb.w);
-  const bool over = gmax > b.zthr;
-  if (h != 0u || over) {
-    uint32_t bits = 0;  // bit k: entry k is a candidate
+  const uint4 cw = philox(x.rk, (uint32_t)base >> 4, x.grow, x.ctr_lo, x.ctr_hi8 | 0u);
+  const bool over = (entry & 16) != 0;
+  // which of the 16 entries need a look (no calls in this loop), then one pass per set bit
+  uint32_t todo = 0;
 #pragma unroll
-    for (int w = 0; w < 4; ++w) {
-      const uint32_t f = ff_bytes(pick_word(cb, w));
-      bits |= (((f >> 7) & 1u) | ((f >> 14) & 2u) | ((f >> 21) & 4u) | ((f >> 28) & 8u)) << (4 * w);
-    }
-    if (over) {
-#pragma unroll
-      for (int k = 0; k < 16; ++k) bits |= (z[k] > b.zthr ? 1u : 0u) << k;
-    }
-    bits &= (1u << valid) - 1u;  // the row may end inside the group
-    while (bits) {
-      const int k = __ffs(bits) - 1;
-      bits &= bits - 1;
-      push_candidate<DT>(x, e0 + k, b, sm, warp);
-    }
+  for (int k = 0; k < 16; ++k) {
+    const uint32_t cbyte = (pick_word(cw, k >> 2) >> (8 * (k & 3))) & 0xFFu;
+    todo |= ((cbyte == 255u || (over && z[k] > b.zthr)) ? 1u : 0u) << k;
   }
+  while (todo) {
+    const int k = __ffs(todo) - 1;
+    todo &= todo - 1;
+    const uint32_t cbyte = (pick_word(cw, k >> 2) >> (8 * (k & 3))) & 0xFFu;
+    eval_element(x, base + k, cbyte, z[k], b, sm);  // padding beyond the row is -inf and drops out there
+  }
+}
+
+template <int DT>
+__device__ __forceinline__ void drain_queue(const EvalCtx &x, Best &b, Smem &sm, int warp, int lane, int &qn,
+                                            bool aligned) {
+  __syncwarp();
+  for (int e = lane; e < qn; e += 32) eval_entry<DT>(x, sm.queue[warp][e], b, sm, aligned);
+  __syncwarp();
+  qn = 0;
+}
+
+// First step of a segment (warp-uniform): a valid lower bound of the row's best score from the coarse
+// byte of each lane's largest entry alone: u >= (c + 2^-33)/256  =>  g >= -ln(ln 256 - ln(c + 2^-33)).
+__device__ __forceinline__ void seed_gate(const EvalCtx &x, const float (&z)[16], float gmax, bool have,
+                                          const uint4 &cb, Best &b, Smem &sm) {
+  float ylo = -CUDART_INF_F;
+  if (have && gmax > -CUDART_INF_F && gmax < CUDART_INF_F) {
+    uint32_t cbyte = 0;
+#pragma unroll
+    for (int k = 15; k >= 0; --k)
+      if (z[k] == gmax) cbyte = (pick_word(cb, k >> 2) >> (8 * (k & 3))) & 0xFFu;
+    const float neg_ln_u = (8.0f - lg2f((float)cbyte + 0x1p-33f)) * kLn2f;
+    const float glo = -lg2f(neg_ln_u) * kLn2f;
+    const float sf = gmax / x.tau;
+    ylo = sf - fabsf(sf) * 2e-6f + glo - 2e-3f;
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) ylo = fmaxf(ylo, __shfl_xor_sync(0xffffffffu, ylo, o));
+  int enc = enc_float(ylo);
+  if ((threadIdx.x & 31) == 0 && enc > enc_neg_inf()) post_best(sm, x.seg, enc);
+  const int cta = read_best(sm, x.seg);
+  enc = enc > cta ? enc : cta;
+  if (enc > b.enc) set_gate(b, enc, x.tau);
+}
+
+// Gate and queue for one group (sampler 0).  qn is the warp's queue fill (warp-uniform).
+__device__ __forceinline__ void sample_group(const EvalCtx &x, float gmax, bool have, int e0, const uint4 &cb, Best &b,
+                                             Smem &sm, int warp, int lane, int &qn) {
+  const uint32_t a0 = any_ff(cb.x), a1 = any_ff(cb.y), a2 = any_ff(cb.z), a3 = any_ff(cb.w);
+  const bool over = have && gmax > b.zthr;
+  const bool flag = (a0 | a1 | a2 | a3) != 0u || over;
+  const uint32_t ballot = __ballot_sync(0xffffffffu, flag);
+  if (ballot != 0u) {
+    if (flag) {
+      const int entry = ((e0 >> 4) << 5) | (over ? 16 : 0) | (a0 ? 1 : 0) | (a1 ? 2 : 0) | (a2 ? 4 : 0) | (a3 ? 8 : 0);
+      sm.queue[warp][qn + __popc(ballot & ((1u << lane) - 1u))] = entry;
+    }
+    qn += __popc(ballot);
+  }
+}
+
+// A consumer thread's running state for the segment it is working on.
+struct LaneState {
+  Acc acc;
+  Best best;
+  int err;
+  int qn;  // fill of the warp's candidate queue (warp-uniform)
+};
+
+// The common case, kept small so that the streaming loop stays in the instruction cache: a full group
+// read from the pipeline stage, finite logits assumed, gate already seeded.
+template <int DT, int SAMPLER>
+__device__ __forceinline__ void hot_group(const EvalCtx &x, const unsigned char *stage, int slot, int e0, float c,
+                                          bool have, Acc &acc, Best &best, int &err, int &qn, Smem &sm, int warp,
+                                          int lane) {
+  float gmax = -CUDART_INF_F;
+  if (have) {
+    RawGroup<DT> raw;
+    load_raw_smem<DT>(stage, slot, raw);
+    float z[16];
+    gmax = unpack_group<DT>(raw, z);
+    accumulate<false>(acc, z, c, gmax, err);
+  }
+  if (SAMPLER == 0) {
+    uint4 cb = make_uint4(0, 0, 0, 0);
+    if (have) cb = philox(x.rk, (uint32_t)e0 >> 4, x.grow, x.ctr_lo, x.ctr_hi8 | 0u);
+    sample_group(x, gmax, have, e0, cb, best, sm, warp, lane, qn);
+  }
+}
+
+// Everything else: the first chunk of a segment (seeds the gate), ragged chunks, rows that do not end on
+// a group boundary, greedy rows, rows that cannot use the ring.  One call handles the thread's group
+// `slot` of the chunk that starts at entry `cs`.
+template <int DT, int SAMPLER>
+__device__ __noinline__ void slow_group(const EvalCtx &x, const unsigned char *stage, int slot, int cs, int e_hi,
+                                        float c, bool greedy, bool seed, LaneState &st, Smem &sm) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int e0 = cs + slot * kGroup;
+  const bool have = e0 < e_hi;
+  const bool full = e0 + kGroup <= x.V;
+  float z[16];
+  float gmax = -CUDART_INF_F;
+  if (have && full && stage != nullptr) {
+    RawGroup<DT> raw;
+    load_raw_smem<DT>(stage, slot, raw);
+    gmax = unpack_group<DT>(raw, z);
+  } else if (have) {
+    gmax = load_group_guarded<DT>(x.row, e0, full ? 16 : x.V - e0, z);
+  } else {
+#pragma unroll
+    for (int k = 0; k < 16; ++k) z[k] = -CUDART_INF_F;
+  }
+  if (greedy) {
+    if (have) {
+      int kk = -1;
+#pragma unroll
+      for (int k = 15; k >= 0; --k) {
+        if (z[k] != z[k] || z[k] == CUDART_INF_F) st.err |= kErrValue;
+        if (z[k] == gmax) kk = k;
+      }
+      if (kk >= 0 && gmax > -CUDART_INF_F && (double)gmax > st.best.y) {
+        st.best.y = (double)gmax;
+        st.best.idx = e0 + kk;
+      }
+    }
+    return;
+  }
+  if (have) {
+    if (full && stage != nullptr)
+      accumulate<false>(st.acc, z, c, gmax, st.err);
+    else
+      accumulate<true>(st.acc, z, c, gmax, st.err);
+  }
+  if (SAMPLER == 0) {
+    uint4 cb = make_uint4(0, 0, 0, 0);
+    if (have) cb = philox(x.rk, (uint32_t)e0 >> 4, x.grow, x.ctr_lo, x.ctr_hi8 | 0u);
+    if (seed) seed_gate(x, z, gmax, have, cb, st.best, sm);
+    sample_group(x, gmax, have, e0, cb, st.best, sm, warp, lane, st.qn);
+  }
+}
+
+// Seeds the gate of sampler 0 from the thread's first group of a segment (full groups read from the
+// stage; other lanes contribute nothing).  Called once per segment, before the streaming loop.
+template <int DT>
+__device__ __noinline__ void seed_from_stage(const EvalCtx &x, const unsigned char *stage, int slot, int e0,
+                                             bool usable, Best &b, Smem &sm) {
+  float z[16];
+  float gmax = -CUDART_INF_F;
+  uint4 cb = make_uint4(0, 0, 0, 0);
+  if (usable) {
+    RawGroup<DT> raw;
+    load_raw_smem<DT>(stage, slot, raw);
+    gmax = unpack_group<DT>(raw, z);
+    cb = philox(x.rk, (uint32_t)e0 >> 4, x.grow, x.ctr_lo, x.ctr_hi8 | 0u);
+  } else {
+#pragma unroll
+    for (int k = 0; k < 16; ++k) z[k] = -CUDART_INF_F;
+  }
+  seed_gate(x, z, gmax, usable, cb, b, sm);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -592,7 +750,8 @@ __global__ void __launch_bounds__(kThreads, 2) rows_kernel(const __grid_constant
   extern __shared__ __align__(128) unsigned char ring[];
   __shared__ Smem sm;
   constexpr int kEsize = DT == 0 ? 4 : 2;
-  constexpr int kStageBytes = kChunk * kEsize;
+  constexpr int kChunkE = kStageBytes / kEsize;                    // entries per stage: 8,192 bf16 / 4,096 fp32
+  constexpr int kGPT = kChunkE / (kStreamThreads * kGroup);        // 16-entry groups per consumer thread and stage
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
   if (tid == 0) {
@@ -602,7 +761,6 @@ __global__ void __launch_bounds__(kThreads, 2) rows_kernel(const __grid_constant
     sm.timeout = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (tid < kStreamWarps) sm.qcount[tid] = 0;
   __syncthreads();
 
   const int full_end = (int)(p.V & ~(int64_t)15);  // entries covered by full groups
@@ -611,76 +769,93 @@ __global__ void __launch_bounds__(kThreads, 2) rows_kernel(const __grid_constant
     // ------------------------------------------------------------------ consumers
     Walker wk(p);
     Seg s;
-    uint32_t cc = 0;   // pipeline chunks consumed so far
-    uint32_t n = 0;    // segments handed to the finishing warp so far
+    uint32_t stage = 0, phase = 0;  // ring position
+    uint32_t n = 0;                 // segments handed to the finishing warp so far
     while (wk.next(p, s)) {
       const RowInfo ri = classify(p, s.row);
       if (ri.skip) continue;
       const char *row = row_ptr<DT>(p, s.row);
       EvalCtx ex;
       ex.rk = p.round_key; ex.row = row; ex.tau = ri.tau; ex.grow = p.row_base + (uint32_t)s.row;
-      ex.ctr_lo = p.ctr_lo; ex.ctr_hi8 = p.ctr_hi8; ex.seg = n + 1;
+      ex.ctr_lo = p.ctr_lo; ex.ctr_hi8 = p.ctr_hi8; ex.seg = n + 1; ex.V = (int)p.V;
 
       Acc acc;
-      acc.R = -CUDART_INF_F; acc.nRc = 0.f; acc.Z0 = acc.Z1 = acc.W0 = acc.W1 = 0.f;
       Best best;
+      int err, qn = 0;
+      acc.R = -CUDART_INF_F; acc.nRc = kNoRef; acc.Z0 = acc.Z1 = acc.W0 = acc.W1 = 0.f;
       best.y = -CUDART_INF; best.idx = -1;
       set_gate(best, enc_neg_inf(), ri.tau);
-      int err = 0;
-      bool seed = SAMPLER == 0 && !ri.greedy;
+      err = 0;
 
-      const int nchunks = s.e_hi > s.e_lo ? (s.e_hi - s.e_lo + kChunk - 1) / kChunk : 0;
+      const int nchunks = s.e_hi > s.e_lo ? (s.e_hi - s.e_lo + kChunkE - 1) / kChunkE : 0;
+      const int fast_end = s.e_hi < full_end ? s.e_hi : full_end;  // chunks ending at or before this are full
+      if (RING && SAMPLER == 0 && !ri.greedy && nchunks > 0) {
+        // seed the gate from the first stage of the segment (the stage is consumed by the loop below)
+        mbar_wait(&sm.full[stage], phase, sm);
+        const int e0 = s.e_lo + tid * kGroup;
+        seed_from_stage<DT>(ex, ring + (size_t)stage * kStageBytes, tid, e0, e0 + kGroup <= fast_end, best, sm);
+      }
+#pragma unroll 1
       for (int c = 0; c < nchunks; ++c) {
-        const int e0 = s.e_lo + c * kChunk + tid * kGroup;
-        const bool have = e0 < s.e_hi;
-        const bool full = e0 + kGroup <= full_end;
-        float z[16];
-        float gmax = -CUDART_INF_F;
+        const int cs = s.e_lo + c * kChunkE;
+        const unsigned char *stage_ptr = nullptr;
         if (RING) {
-          const uint32_t stage = cc % kStages, round = cc / kStages;
-          mbar_wait(&sm.full[stage], round & 1u, sm);
-          if (have && full) gmax = load_group_smem<DT>(ring + (size_t)stage * kStageBytes, tid, z);
+          mbar_wait(&sm.full[stage], phase, sm);
+          stage_ptr = ring + (size_t)stage * kStageBytes;
+        }
+        if (SAMPLER == 0 && !ri.greedy) {
+          const int enc = read_best(sm, ex.seg);
+          if (enc > best.enc) set_gate(best, enc, ri.tau);
+        }
+        if (RING && !ri.greedy) {
+          const bool all_full = cs + kChunkE <= fast_end;
+#pragma unroll
+          for (int j = 0; j < kGPT; ++j) {
+            const int slot = j * kStreamThreads + tid;
+            const int e0 = cs + slot * kGroup;
+            hot_group<DT, SAMPLER>(ex, stage_ptr, slot, e0, ri.c, all_full || e0 + kGroup <= fast_end, acc, best, err,
+                                   qn, sm, warp, lane);
+          }
+          // the row's last, partial group (V not a multiple of 16) goes through the out-of-line path
+          if (!all_full && fast_end < s.e_hi && fast_end >= cs && fast_end < cs + kChunkE) {
+            const int slot = (fast_end - cs) / kGroup;
+            if (((slot % kStreamThreads) >> 5) == warp) {
+              LaneState st;
+              st.acc = acc; st.best = best; st.err = err; st.qn = qn;
+              // only the owning lane has the group; the others pass an empty range
+              slow_group<DT, SAMPLER>(ex, nullptr, slot, cs, (slot % kStreamThreads) == tid ? s.e_hi : 0, ri.c, false,
+                                      false, st, sm);
+              acc = st.acc; best = st.best; err = st.err; qn = st.qn;
+            }
+          }
+        } else {
+          // the out-of-line path works on a copy, so that the streaming loop keeps its state in registers
+          LaneState st;
+          st.acc = acc; st.best = best; st.err = err; st.qn = qn;
+#pragma unroll 1
+          for (int j = 0; j < kGPT; ++j)
+            slow_group<DT, SAMPLER>(ex, stage_ptr, j * kStreamThreads + tid, cs, s.e_hi, ri.c, ri.greedy,
+                                    !RING && SAMPLER == 0 && !ri.greedy && c == 0 && j == 0, st, sm);
+          acc = st.acc; best = st.best; err = st.err; qn = st.qn;
+        }
+        if (RING) {
           __syncwarp();
           if (lane == 0) mbar_arrive(&sm.empty[stage]);
-          ++cc;
-          if (have && !full) gmax = load_group_guarded<DT>(row, e0, (int)p.V - e0, z);
-        } else if (have) {
-          gmax = load_group_guarded<DT>(row, e0, full ? 16 : (int)p.V - e0, z);
+          if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
-        if (ri.greedy) {
-          if (have) {
-            int kk = -1;
-#pragma unroll
-            for (int k = 15; k >= 0; --k) {
-              if (z[k] != z[k] || z[k] == CUDART_INF_F) err |= kErrValue;
-              if (z[k] == gmax) kk = k;
-            }
-            if (kk >= 0 && gmax > -CUDART_INF_F && (double)gmax > best.y) { best.y = (double)gmax; best.idx = e0 + kk; }
-          }
-          continue;
-        }
-        if (have) {
-          if (full)
-            accumulate<false>(acc, z, ri.c, gmax, err);
-          else
-            accumulate<true>(acc, z, ri.c, gmax, err);
-        }
-        if (SAMPLER == 0) {
-          sample_group<DT>(ex, z, gmax, have, e0, full ? 16 : (int)p.V - e0, best, sm, warp, seed);
-          seed = false;
-          drain_queue<DT>(ex, best, sm, warp, lane, kDrainAt);
-        }
+        if (SAMPLER == 0 && qn >= kDrainAt) drain_queue<DT>(ex, best, sm, warp, lane, qn, RING);
       }
-      if (SAMPLER == 0 && !ri.greedy) drain_queue<DT>(ex, best, sm, warp, lane, 1);
+      if (SAMPLER == 0 && qn > 0) drain_queue<DT>(ex, best, sm, warp, lane, qn, RING);
 
       if (!ri.greedy) {
         // -inf or NaN logits poison the fast sums: redo this warp's groups with the careful form
         const float zs = acc.Z0 + acc.Z1, ws = acc.W0 + acc.W1;
         const bool bad = !(fabsf(zs) < CUDART_INF_F) || !(fabsf(ws) < CUDART_INF_F);
         if (__any_sync(0xffffffffu, bad)) {
-          acc.R = -CUDART_INF_F; acc.nRc = 0.f; acc.Z0 = acc.Z1 = acc.W0 = acc.W1 = 0.f;
-          for (int c = 0; c < nchunks; ++c) {
-            const int e0 = s.e_lo + c * kChunk + tid * kGroup;
+          acc.R = -CUDART_INF_F; acc.nRc = kNoRef; acc.Z0 = acc.Z1 = acc.W0 = acc.W1 = 0.f;
+#pragma unroll 1
+          for (int c = 0; c < nchunks * kGPT; ++c) {
+            const int e0 = s.e_lo + (c * kStreamThreads + tid) * kGroup;
             if (e0 < s.e_hi) {
               float z[16];
               const float gmax = load_group_guarded<DT>(row, e0, e0 + kGroup <= (int)p.V ? 16 : (int)p.V - e0, z);
@@ -719,18 +894,17 @@ __global__ void __launch_bounds__(kThreads, 2) rows_kernel(const __grid_constant
     if (RING && lane == 0) {
       Walker wk(p);
       Seg s;
-      uint32_t cc = 0;
+      uint32_t cc = 0, stage = 0, phase = 1;  // phase: parity of the previous use of the stage
       while (wk.next(p, s)) {
         const RowInfo ri = classify(p, s.row);
         if (ri.skip) continue;
         const char *row = row_ptr<DT>(p, s.row);
-        const int nchunks = s.e_hi > s.e_lo ? (s.e_hi - s.e_lo + kChunk - 1) / kChunk : 0;
+        const int nchunks = s.e_hi > s.e_lo ? (s.e_hi - s.e_lo + kChunkE - 1) / kChunkE : 0;
         const int lim = s.e_hi < full_end ? s.e_hi : full_end;
         for (int c = 0; c < nchunks; ++c) {
-          const uint32_t stage = cc % kStages, round = cc / kStages;
-          if (round > 0) mbar_wait(&sm.empty[stage], (round - 1) & 1u, sm);
-          const int cs = s.e_lo + c * kChunk;
-          const int ce = cs + kChunk < lim ? cs + kChunk : lim;
+          if (cc >= (uint32_t)kStages) mbar_wait(&sm.empty[stage], phase, sm, 64u);
+          const int cs = s.e_lo + c * kChunkE;
+          const int ce = cs + kChunkE < lim ? cs + kChunkE : lim;
           const uint32_t bytes = ce > cs ? (uint32_t)(ce - cs) * kEsize : 0u;
           const bool dead = *reinterpret_cast<volatile int *>(&sm.timeout) != 0;
           if (bytes > 0 && !dead) {
@@ -740,6 +914,7 @@ __global__ void __launch_bounds__(kThreads, 2) rows_kernel(const __grid_constant
             mbar_arrive(&sm.full[stage]);
           }
           ++cc;
+          if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
       }
       // Before leaving, see every copy still in flight land (bounded).
@@ -762,7 +937,7 @@ __global__ void __launch_bounds__(kThreads, 2) rows_kernel(const __grid_constant
         continue;
       }
       const uint32_t slot = n % kSlots, use = n / kSlots;
-      mbar_wait(&sm.wfull[slot], use & 1u, sm);
+      mbar_wait_warp(&sm.wfull[slot], use & 1u, sm, lane);
       double Md = 0.0, Zd = 0.0, Wd = 0.0, yd = -CUDART_INF;
       int id = -1, ed = 0;
       if (lane < kStreamWarps) {
@@ -839,7 +1014,7 @@ cudaError_t setup_kernel(KernelSetup &out) {
   std::lock_guard<std::mutex> hold(lock);
   if (cache[dev].ctas_per_sm == 0) {
     auto kern = rows_kernel<DT, SAMPLER, RING>;
-    const size_t dyn = RING ? (size_t)kStages * kChunk * (DT == 0 ? 4 : 2) : 0;
+    const size_t dyn = RING ? (size_t)kStages * kStageBytes : 0;
     e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn);
     if (e != cudaSuccess) return e;
     KernelSetup ks;
@@ -883,7 +1058,7 @@ cudaError_t launch_one(RowsParams p, void *workspace, size_t workspace_bytes, cu
     p.ws_arrivals = reinterpret_cast<unsigned long long *>(p.ws_pieces + (size_t)kMaxGrid * 2 * kPieceBytes);
   }
   p.call_id = next_call_id();
-  const size_t dyn = RING ? (size_t)kStages * kChunk * (DT == 0 ? 4 : 2) : 0;
+  const size_t dyn = RING ? (size_t)kStages * kStageBytes : 0;
   rows_kernel<DT, SAMPLER, RING><<<(unsigned)grid, kThreads, dyn, stream>>>(p);
   return cudaGetLastError();
 }

@@ -11,7 +11,7 @@ constexpr int kStreamThreads = kStreamWarps * 32;   // 256
 constexpr int kThreads = kStreamThreads + 64;       // + one warp that issues bulk copies + one that finishes rows
 constexpr int kGroup = 16;                          // vocabulary entries per coarse Philox call
 constexpr int kTile = 512;                          // unit of the work split (entries); CTA ranges start on tile bounds
-constexpr int kChunk = 4096;                        // entries per pipeline stage (one 16-entry group per consumer thread)
+constexpr int kStageBytes = 16384;                   // bytes per pipeline stage (one bulk copy)
 constexpr int kStages = 6;
 constexpr int kMaxGrid = 1024;                      // CTAs the piece workspace is sized for
 constexpr size_t kPieceBytes = 64;                  // one partial row state in the workspace
