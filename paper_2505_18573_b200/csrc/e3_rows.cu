@@ -42,8 +42,8 @@
 namespace e3 {
 namespace {
 
-constexpr int kQueueCap = 96;
-constexpr int kDrainAt = 32;
+constexpr int kQueueCap = 192;
+constexpr int kDrainEvery = 4;  // chunks between drains (power of two)
 constexpr int kSlots = 4;  // hand-over slots between the consumer warps and the finishing warp
 constexpr uint32_t kSpinLimit = 1u << 23;  // polls before a wait gives up (seconds)
 constexpr float kLog2e = 1.4426950408889634f;
@@ -61,7 +61,8 @@ struct Piece {  // one partial row state in the workspace (kPieceBytes)
   double y;        // best perturbed score (greedy rows: largest logit)
   int idx;         // its vocabulary index, -1 = none
   int err;
-  int pad[6];
+  float ty[3];     // sampler 1: the three best block scores (fp32) ...
+  int tb[3];       // ... and their block indices, -1 = none
 };
 static_assert(sizeof(Piece) == kPieceBytes, "piece size");
 
@@ -70,6 +71,8 @@ struct WarpPartial {
   int idx;
   double y;
   int err;
+  float ty[3];
+  int tb[3];
   int pad;
 };
 
@@ -164,7 +167,7 @@ __device__ __forceinline__ void mbar_wait(unsigned long long *b, uint32_t parity
 }
 // Whole-warp wait with a single polling lane (used by the finishing warp, which mostly waits).
 __device__ __forceinline__ void mbar_wait_warp(unsigned long long *b, uint32_t parity, Smem &sm, int lane) {
-  if (lane == 0) mbar_wait(b, parity, sm, 512u);
+  if (lane == 0) mbar_wait(b, parity, sm, 2000u);
   __syncwarp();
 }
 __device__ __forceinline__ void bulk_copy_g2s(void *dst, const void *src, uint32_t bytes, unsigned long long *bar) {
@@ -605,6 +608,173 @@ __device__ __noinline__ void seed_from_stage(const EvalCtx &x, const unsigned ch
 }
 
 // ---------------------------------------------------------------------------------------------
+// Sampler 1: one Gumbel per block of 256 consecutive entries, applied to the block's log-sum-exp.
+// A block is 16 consecutive groups, i.e. one half-warp in one step.  All lanes of a warp keep the
+// same reference (the warp-wide largest logit so far), so that the 16 group sums of a block add up
+// directly.  Each half-warp parks one block sum per step in one of its lanes; every 16 steps all
+// lanes turn their parked block into a score Y_b = L_b + g_b (one Philox call and three MUFU each)
+// and keep the three best (fp32).  The finishing warp settles near-ties in fp64 and draws the
+// token inside the winning block by inverse CDF.
+// ---------------------------------------------------------------------------------------------
+struct Top3 {
+  float y[3];
+  int b[3];
+};
+__device__ __forceinline__ void top3_reset(Top3 &t) {
+  t.y[0] = t.y[1] = t.y[2] = -CUDART_INF_F;
+  t.b[0] = t.b[1] = t.b[2] = -1;
+}
+// order: larger score first, equal scores by lower block index; NaN scores never enter
+__device__ __forceinline__ bool top3_before(float y, int b, float y2, int b2) {
+  return b2 < 0 || y > y2 || (y == y2 && b < b2);
+}
+__device__ __forceinline__ void top3_insert(Top3 &t, float y, int b) {
+  if (b < 0 || !(y == y)) return;
+  if (top3_before(y, b, t.y[0], t.b[0])) {
+    t.y[2] = t.y[1]; t.b[2] = t.b[1]; t.y[1] = t.y[0]; t.b[1] = t.b[0]; t.y[0] = y; t.b[0] = b;
+  } else if (top3_before(y, b, t.y[1], t.b[1])) {
+    t.y[2] = t.y[1]; t.b[2] = t.b[1]; t.y[1] = y; t.b[1] = b;
+  } else if (top3_before(y, b, t.y[2], t.b[2])) {
+    t.y[2] = y; t.b[2] = b;
+  }
+}
+__device__ __forceinline__ void top3_merge(Top3 &t, const Top3 &o) {
+#pragma unroll
+  for (int i = 0; i < 3; ++i) top3_insert(t, o.y[i], o.b[i]);
+}
+
+struct BlockState {
+  Top3 top;
+  float S, ref;  // parked block: sum 2^(z c + ref)
+  int b;         // its block index
+  int it;        // steps taken in this segment (warp-uniform)
+};
+__device__ __forceinline__ void block_state_reset(BlockState &bs) {
+  top3_reset(bs.top);
+  bs.S = 0.f; bs.ref = 0.f; bs.b = -1; bs.it = 0;
+}
+
+// fp32 Gumbel variate of block b: u = (x + 1/2) 2^-32, g = -ln(-ln u)
+__device__ __forceinline__ float block_gumbel_f32(const EvalCtx &x, int b) {
+  const uint4 w = philox(x.rk, (uint32_t)b >> 2, x.grow, x.ctr_lo, x.ctr_hi8 | 2u);
+  const uint32_t xw = pick_word(w, b & 3);
+  float a;  // -ln u
+  if (xw >= 0xFE000000u) {
+    const float d = ((float)(~xw) + 0.5f) * 0x1p-32f;  // 1 - u < 2^-7: series of -ln(1 - d)
+    a = d * fmaf(d, fmaf(d, 0.33333334f, 0.5f), 1.0f);
+  } else {
+    a = -lg2f(((float)xw + 0.5f) * 0x1p-32f) * kLn2f;
+  }
+  return -lg2f(a) * kLn2f;
+}
+
+__device__ __forceinline__ void block_flush(const EvalCtx &x, BlockState &bs) {
+  if (bs.b >= 0 && bs.S > 0.f) {
+    const float L = (lg2f(bs.S) - bs.ref) * kLn2f;  // ln sum_i exp(s_i) over the block
+    top3_insert(bs.top, L + block_gumbel_f32(x, bs.b), bs.b);
+  }
+  bs.S = 0.f;
+  bs.b = -1;
+}
+
+// One step of a warp: every lane brings (at most) one group.  CAREFUL lanes skip -inf / NaN entries.
+template <bool CAREFUL>
+__device__ __forceinline__ void block_step(const EvalCtx &x, const float (&z)[16], float gmax, bool have, int e0,
+                                           float c, Acc &a, BlockState &bs, int &err, int lane) {
+  if (CAREFUL && have && gmax == CUDART_INF_F) err |= kErrValue;
+  const int mw = __reduce_max_sync(0xffffffffu, enc_float(have ? gmax : -CUDART_INF_F));
+  if (mw != enc_neg_inf()) {  // warp-uniform
+    const float R = fmaxf(a.R, dec_float(mw));
+    const float nRc = -R * c;
+    const float d = nRc - a.nRc;
+    const float f = ex2f(d);
+    a.W0 = f * fmaf(d, a.Z0, a.W0);
+    a.W1 = f * fmaf(d, a.Z1, a.W1);
+    a.Z0 *= f;
+    a.Z1 *= f;
+    a.R = R;
+    a.nRc = nRc;
+    float g0 = 0.f, g1 = 0.f;
+    if (have) {
+#pragma unroll
+      for (int k = 0; k < 16; k += 2) {
+        if (CAREFUL) {
+          if (z[k] != z[k] || z[k + 1] != z[k + 1]) err |= kErrValue;
+          if (z[k] != -CUDART_INF_F && z[k] == z[k]) {
+            const float t = fmaf(z[k], c, nRc), e = ex2f(t);
+            g0 += e;
+            a.W0 = fmaf(e, t, a.W0);
+          }
+          if (z[k + 1] != -CUDART_INF_F && z[k + 1] == z[k + 1]) {
+            const float t = fmaf(z[k + 1], c, nRc), e = ex2f(t);
+            g1 += e;
+            a.W1 = fmaf(e, t, a.W1);
+          }
+        } else {
+          const float t0 = fmaf(z[k], c, nRc), t1 = fmaf(z[k + 1], c, nRc);
+          const float e0_ = ex2f(t0), e1_ = ex2f(t1);
+          g0 += e0_;
+          g1 += e1_;
+          a.W0 = fmaf(e0_, t0, a.W0);
+          a.W1 = fmaf(e1_, t1, a.W1);
+        }
+      }
+      a.Z0 += g0;
+      a.Z1 += g1;
+    }
+    float sb = g0 + g1;
+#pragma unroll
+    for (int o = 1; o < 16; o <<= 1) sb += __shfl_xor_sync(0xffffffffu, sb, o);
+    if ((bs.it & 15) == (lane & 15)) {
+      bs.S = sb;
+      bs.ref = nRc;
+      bs.b = e0 >> 8;
+    }
+  }
+  ++bs.it;
+  if ((bs.it & 15) == 0) block_flush(x, bs);
+}
+
+template <int DT>
+__device__ __forceinline__ void hot_group_blocks(const EvalCtx &x, const unsigned char *stage, int slot, int e0,
+                                                 float c, Acc &acc, BlockState &bs, int &err, int lane) {
+  RawGroup<DT> raw;
+  load_raw_smem<DT>(stage, slot, raw);
+  float z[16];
+  const float gmax = unpack_group<DT>(raw, z);
+  block_step<false>(x, z, gmax, true, e0, c, acc, bs, err, lane);
+}
+
+struct LaneStateBlocks {
+  Acc acc;
+  BlockState bs;
+  int err;
+};
+
+// Out-of-line form: ragged chunks, the row's partial last group, rows that cannot use the ring.
+template <int DT>
+__device__ __noinline__ void slow_group_blocks(const EvalCtx &x, const unsigned char *stage, int slot, int cs,
+                                               int e_hi, float c, LaneStateBlocks &st) {
+  const int lane = threadIdx.x & 31;
+  const int e0 = cs + slot * kGroup;
+  const bool have = e0 < e_hi;
+  const bool full = e0 + kGroup <= x.V;
+  float z[16];
+  float gmax = -CUDART_INF_F;
+  if (have && full && stage != nullptr) {
+    RawGroup<DT> raw;
+    load_raw_smem<DT>(stage, slot, raw);
+    gmax = unpack_group<DT>(raw, z);
+  } else if (have) {
+    gmax = load_group_guarded<DT>(x.row, e0, full ? 16 : x.V - e0, z);
+  } else {
+#pragma unroll
+    for (int k = 0; k < 16; ++k) z[k] = -CUDART_INF_F;
+  }
+  block_step<true>(x, z, gmax, have, e0, c, st.acc, st.bs, st.err, lane);
+}
+
+// ---------------------------------------------------------------------------------------------
 // Merging partial states
 // ---------------------------------------------------------------------------------------------
 __device__ __forceinline__ void merge_stats_f(float &M, float &Z, float &W, float M2, float Z2, float W2) {
@@ -743,6 +913,116 @@ __device__ __forceinline__ void write_skipped(const RowsParams &p, int64_t row, 
 }
 
 // ---------------------------------------------------------------------------------------------
+// Sampler 1, finishing warp: exact (fp64) block scores where fp32 cannot separate the leaders, then the
+// in-block inverse-CDF draw.  All 32 lanes take part; a block is 8 consecutive entries per lane.
+// ---------------------------------------------------------------------------------------------
+struct BlockView {
+  double s[8];  // z/tau of the lane's entries (-inf beyond the row)
+  double m;     // block maximum
+};
+
+template <int DT>
+__device__ __forceinline__ void load_block(const char *row, int b, int V, double tau, int lane, BlockView &v) {
+  double m = -CUDART_INF;
+#pragma unroll
+  for (int k = 0; k < 8; ++k) {
+    const int i = b * 256 + lane * 8 + k;
+    const float z = i < V ? load_elem<DT>(row, i) : -CUDART_INF_F;
+    v.s[k] = (double)z / tau;
+    m = fmax(m, v.s[k]);
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) m = fmax(m, __shfl_xor_sync(0xffffffffu, m, o));
+  v.m = m;
+}
+
+// Y_b = m_b + ln sum exp(s_i - m_b) + g_b in fp64; -inf for a block without mass.
+template <int DT>
+__device__ __noinline__ double exact_block_score(const EvalCtx &x, int b, int lane) {
+  BlockView v;
+  load_block<DT>(x.row, b, x.V, (double)x.tau, lane, v);
+  if (v.m == -CUDART_INF) return -CUDART_INF;
+  double sum = 0.0;
+#pragma unroll
+  for (int k = 0; k < 8; ++k)
+    if (v.s[k] != -CUDART_INF) sum += exp(v.s[k] - v.m);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+  const uint4 w = philox(x.rk, (uint32_t)b >> 2, x.grow, x.ctr_lo, x.ctr_hi8 | 2u);
+  const double u = ((double)pick_word(w, b & 3) + 0.5) * 0x1p-32;
+  return v.m + log(sum) + (-log(-log(u)));
+}
+
+// Token inside block b: first entry whose inclusive prefix sum of exp(s_i - m_b) exceeds v * total.
+template <int DT>
+__device__ __noinline__ int draw_in_block(const EvalCtx &x, int b, int lane) {
+  BlockView v;
+  load_block<DT>(x.row, b, x.V, (double)x.tau, lane, v);
+  double pre[8];
+  double run = 0.0;
+  int last_nonzero = -1;
+#pragma unroll
+  for (int k = 0; k < 8; ++k) {
+    const double w = (v.s[k] != -CUDART_INF) ? exp(v.s[k] - v.m) : 0.0;
+    if (w > 0.0) last_nonzero = k;
+    run += w;
+    pre[k] = run;
+  }
+  double incl = run;  // inclusive scan of the lane totals
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const double up = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += up;
+  }
+  const double total = __shfl_sync(0xffffffffu, incl, 31);
+  const double before = incl - run;
+  const uint4 w3 = philox(x.rk, 0u, x.grow, x.ctr_lo, x.ctr_hi8 | 3u);
+  const double t = (((double)w3.x + 0.5) * 0x1p-32) * total;
+  int hit = -1;
+#pragma unroll
+  for (int k = 7; k >= 0; --k)
+    if (before + pre[k] > t) hit = k;
+  const uint32_t found = __ballot_sync(0xffffffffu, hit >= 0);
+  int tok;
+  if (found != 0u) {
+    const int src = __ffs(found) - 1;
+    tok = b * 256 + src * 8 + __shfl_sync(0xffffffffu, hit, src);
+  } else {  // rounding left t at or above the total: last entry that carries mass
+    const uint32_t any = __ballot_sync(0xffffffffu, last_nonzero >= 0);
+    if (any == 0u) return -1;
+    const int src = 31 - __clz(any);
+    tok = b * 256 + src * 8 + __shfl_sync(0xffffffffu, last_nonzero, src);
+  }
+  return tok;
+}
+
+// Picks the winning block from the three fp32 leaders (exact scores where they are too close) and
+// draws the token.  Returns -1 when the row has no block with mass.
+template <int DT>
+__device__ __noinline__ int sample_in_blocks(const EvalCtx &x, const Top3 &top, int lane) {
+  if (top.b[0] < 0) return -1;
+  int bstar = top.b[0];
+  const float margin = 1e-4f + 2e-5f * fabsf(top.y[0]);
+  if (top.b[1] >= 0 && top.y[0] - top.y[1] <= margin) {
+    double ybest = -CUDART_INF;
+    int bbest = -1;
+    if (top.b[2] >= 0 && top.y[0] - top.y[2] <= margin) {
+      const int nb = (x.V + 255) / 256;  // more than two contenders: settle all blocks exactly
+      for (int b = 0; b < nb; ++b) {
+        const double y = exact_block_score<DT>(x, b, lane);
+        if (y > ybest) { ybest = y; bbest = b; }
+      }
+    } else {
+      const int lo = top.b[0] < top.b[1] ? top.b[0] : top.b[1], hi = top.b[0] < top.b[1] ? top.b[1] : top.b[0];
+      const double y0 = exact_block_score<DT>(x, lo, lane), y1 = exact_block_score<DT>(x, hi, lane);
+      bbest = y1 > y0 ? hi : lo;
+    }
+    if (bbest >= 0) bstar = bbest;
+  }
+  return draw_in_block<DT>(x, bstar, lane);
+}
+
+// ---------------------------------------------------------------------------------------------
 // The kernel
 // ---------------------------------------------------------------------------------------------
 template <int DT, int SAMPLER, bool RING>
@@ -786,6 +1066,8 @@ __global__ void __launch_bounds__(kThreads, 2) rows_kernel(const __grid_constant
       best.y = -CUDART_INF; best.idx = -1;
       set_gate(best, enc_neg_inf(), ri.tau);
       err = 0;
+      BlockState bs;
+      block_state_reset(bs);
 
       const int nchunks = s.e_hi > s.e_lo ? (s.e_hi - s.e_lo + kChunkE - 1) / kChunkE : 0;
       const int fast_end = s.e_hi < full_end ? s.e_hi : full_end;  // chunks ending at or before this are full
@@ -807,7 +1089,22 @@ __global__ void __launch_bounds__(kThreads, 2) rows_kernel(const __grid_constant
           const int enc = read_best(sm, ex.seg);
           if (enc > best.enc) set_gate(best, enc, ri.tau);
         }
-        if (RING && !ri.greedy) {
+        if (SAMPLER == 1 && !ri.greedy) {
+          if (RING && cs + kChunkE <= fast_end) {
+#pragma unroll
+            for (int j = 0; j < kGPT; ++j) {
+              const int slot = j * kStreamThreads + tid;
+              hot_group_blocks<DT>(ex, stage_ptr, slot, cs + slot * kGroup, ri.c, acc, bs, err, lane);
+            }
+          } else {
+            LaneStateBlocks st;
+            st.acc = acc; st.bs = bs; st.err = err;
+#pragma unroll 1
+            for (int j = 0; j < kGPT; ++j)
+              slow_group_blocks<DT>(ex, stage_ptr, j * kStreamThreads + tid, cs, s.e_hi, ri.c, st);
+            acc = st.acc; bs = st.bs; err = st.err;
+          }
+        } else if (RING && !ri.greedy) {
           const bool all_full = cs + kChunkE <= fast_end;
 #pragma unroll
           for (int j = 0; j < kGPT; ++j) {
@@ -843,9 +1140,13 @@ __global__ void __launch_bounds__(kThreads, 2) rows_kernel(const __grid_constant
           if (lane == 0) mbar_arrive(&sm.empty[stage]);
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
-        if (SAMPLER == 0 && qn >= kDrainAt) drain_queue<DT>(ex, best, sm, warp, lane, qn, RING);
+        // All warps of the CTA drain at the same chunks: a drain stalls its warp for microseconds and the
+        // ring moves at the pace of the slowest warp, so staggered drains would add up.
+        if (SAMPLER == 0 && qn > 0 && ((c & (kDrainEvery - 1)) == kDrainEvery - 1 || qn > kQueueCap - 32 * kGPT))
+          drain_queue<DT>(ex, best, sm, warp, lane, qn, RING);
       }
       if (SAMPLER == 0 && qn > 0) drain_queue<DT>(ex, best, sm, warp, lane, qn, RING);
+      if (SAMPLER == 1 && !ri.greedy) block_flush(ex, bs);
 
       if (!ri.greedy) {
         // -inf or NaN logits poison the fast sums: redo this warp's groups with the careful form
@@ -879,12 +1180,23 @@ __global__ void __launch_bounds__(kThreads, 2) rows_kernel(const __grid_constant
         err |= __shfl_xor_sync(0xffffffffu, err, o);
         merge_stats_f(M, Z, W, M2, Z2, W2);
         merge_best(y, idx, y2, idx2);
+        if (SAMPLER == 1) {
+          Top3 o2;
+#pragma unroll
+          for (int i = 0; i < 3; ++i) {
+            o2.y[i] = __shfl_xor_sync(0xffffffffu, bs.top.y[i], o);
+            o2.b[i] = __shfl_xor_sync(0xffffffffu, bs.top.b[i], o);
+          }
+          top3_merge(bs.top, o2);
+        }
       }
       const uint32_t slot = n % kSlots, use = n / kSlots;
       if (use > 0) mbar_wait(&sm.wfree[slot], (use - 1) & 1u, sm);
       if (lane == 0) {
         WarpPartial &w = sm.wpart[slot][warp];
         w.M = M; w.Z = Z; w.W = W; w.y = y; w.idx = idx; w.err = err;
+#pragma unroll
+        for (int i = 0; i < 3; ++i) { w.ty[i] = bs.top.y[i]; w.tb[i] = bs.top.b[i]; }
         mbar_arrive(&sm.wfull[slot]);
       }
       ++n;
@@ -902,7 +1214,7 @@ __global__ void __launch_bounds__(kThreads, 2) rows_kernel(const __grid_constant
         const int nchunks = s.e_hi > s.e_lo ? (s.e_hi - s.e_lo + kChunkE - 1) / kChunkE : 0;
         const int lim = s.e_hi < full_end ? s.e_hi : full_end;
         for (int c = 0; c < nchunks; ++c) {
-          if (cc >= (uint32_t)kStages) mbar_wait(&sm.empty[stage], phase, sm, 64u);
+          if (cc >= (uint32_t)kStages) mbar_wait(&sm.empty[stage], phase, sm, 200u);
           const int cs = s.e_lo + c * kChunkE;
           const int ce = cs + kChunkE < lim ? cs + kChunkE : lim;
           const uint32_t bytes = ce > cs ? (uint32_t)(ce - cs) * kEsize : 0u;
@@ -940,9 +1252,15 @@ __global__ void __launch_bounds__(kThreads, 2) rows_kernel(const __grid_constant
       mbar_wait_warp(&sm.wfull[slot], use & 1u, sm, lane);
       double Md = 0.0, Zd = 0.0, Wd = 0.0, yd = -CUDART_INF;
       int id = -1, ed = 0;
+      Top3 top;
+      top3_reset(top);
       if (lane < kStreamWarps) {
         const WarpPartial &w = sm.wpart[slot][lane];
         Md = w.M; Zd = w.Z; Wd = w.W; yd = w.y; id = w.idx; ed = w.err;
+        if (SAMPLER == 1) {
+#pragma unroll
+          for (int i = 0; i < 3; ++i) { top.y[i] = w.ty[i]; top.b[i] = w.tb[i]; }
+        }
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(&sm.wfree[slot]);
@@ -955,42 +1273,76 @@ __global__ void __launch_bounds__(kThreads, 2) rows_kernel(const __grid_constant
         ed |= __shfl_xor_sync(0xffffffffu, ed, o);
         merge_stats_d(Md, Zd, Wd, M2, Z2, W2);
         merge_best(yd, id, y2, i2);
+        if (SAMPLER == 1) {
+          Top3 o2;
+#pragma unroll
+          for (int i = 0; i < 3; ++i) {
+            o2.y[i] = __shfl_xor_sync(0xffffffffu, top.y[i], o);
+            o2.b[i] = __shfl_xor_sync(0xffffffffu, top.b[i], o);
+          }
+          top3_merge(top, o2);
+        }
       }
-      if (lane != 0) continue;
-      if (*reinterpret_cast<volatile int *>(&sm.timeout)) ed |= kErrTimeout;
-      if (s.whole) {
-        finish_row<DT>(p, s.row, ri, Md, Zd, Wd, yd, id, ed);
-        continue;
+      // lane 0 runs the piece protocol and decides whether this CTA finishes the row
+      int fin = 0;
+      if (lane == 0) {
+        if (*reinterpret_cast<volatile int *>(&sm.timeout)) ed |= kErrTimeout;
+        if (s.whole) {
+          fin = 1;
+        } else {
+          // A piece of a cut row: store it, announce it; whoever completes the row finishes it.
+          Piece *mine = pieces + (size_t)blockIdx.x * 2 + (s.first ? 0 : 1);
+          mine->M = Md; mine->Z = Zd; mine->W = Wd; mine->y = yd; mine->idx = id; mine->err = ed;
+#pragma unroll
+          for (int i = 0; i < 3; ++i) { mine->ty[i] = top.y[i]; mine->tb[i] = top.b[i]; }
+          __threadfence();
+          const unsigned long long tag = p.call_id << 16;
+          unsigned long long *word = p.ws_arrivals + s.k0;
+          unsigned long long cur = *reinterpret_cast<volatile unsigned long long *>(word), want = 0;
+          bool done = false;
+          for (int it = 0; it < 65536 && !done; ++it) {  // lock-free: some contender always gets through
+            want = (cur >> 16) == p.call_id ? cur + 1 : (tag | 1ull);
+            const unsigned long long prev = atomicCAS(word, cur, want);
+            done = prev == cur;
+            cur = prev;
+          }
+          if (done && (int)(want & 0xFFFFull) == s.k1 - s.k0 + 1) {  // the last piece of the row
+            __threadfence();
+            Md = 0.0; Zd = 0.0; Wd = 0.0; yd = -CUDART_INF; id = -1; ed = 0;
+            top3_reset(top);
+            for (int k = s.k0; k <= s.k1; ++k) {
+              // CTA k keeps this row's piece in slot 0 when the row is the first thing it works on
+              const bool is_first_seg = first_tile_of(p, k) / p.tiles_per_row == s.row;
+              const volatile Piece *q = pieces + (size_t)k * 2 + (is_first_seg ? 0 : 1);
+              const double M2 = q->M, Z2 = q->Z, W2 = q->W, y2 = q->y;
+              const int i2 = q->idx;
+              ed |= q->err;
+              merge_stats_d(Md, Zd, Wd, M2, Z2, W2);
+              merge_best(yd, id, y2, i2);
+              if (SAMPLER == 1) {
+#pragma unroll
+                for (int i = 0; i < 3; ++i) top3_insert(top, q->ty[i], q->tb[i]);
+              }
+            }
+            fin = 1;
+          }
+        }
       }
-      // A piece of a cut row: store it, announce it; whoever completes the row finishes it.
-      Piece *mine = pieces + (size_t)blockIdx.x * 2 + (s.first ? 0 : 1);
-      mine->M = Md; mine->Z = Zd; mine->W = Wd; mine->y = yd; mine->idx = id; mine->err = ed;
-      __threadfence();
-      const unsigned long long tag = p.call_id << 16;
-      unsigned long long *word = p.ws_arrivals + s.k0;
-      unsigned long long cur = *reinterpret_cast<volatile unsigned long long *>(word), want = 0;
-      bool done = false;
-      for (int it = 0; it < 65536 && !done; ++it) {  // lock-free: some contender always gets through
-        want = (cur >> 16) == p.call_id ? cur + 1 : (tag | 1ull);
-        const unsigned long long prev = atomicCAS(word, cur, want);
-        done = prev == cur;
-        cur = prev;
+      fin = __shfl_sync(0xffffffffu, fin, 0);
+      if (!fin) continue;
+      if (SAMPLER == 1 && !ri.greedy) {
+        // the whole warp settles the block and draws inside it
+#pragma unroll
+        for (int i = 0; i < 3; ++i) {
+          top.y[i] = __shfl_sync(0xffffffffu, top.y[i], 0);
+          top.b[i] = __shfl_sync(0xffffffffu, top.b[i], 0);
+        }
+        EvalCtx ex;
+        ex.rk = p.round_key; ex.row = row_ptr<DT>(p, s.row); ex.tau = ri.tau; ex.grow = p.row_base + (uint32_t)s.row;
+        ex.ctr_lo = p.ctr_lo; ex.ctr_hi8 = p.ctr_hi8; ex.seg = 0; ex.V = (int)p.V;
+        id = sample_in_blocks<DT>(ex, top, lane);
       }
-      if (!done || (int)(want & 0xFFFFull) != s.k1 - s.k0 + 1) continue;  // not the last piece of the row
-      __threadfence();
-      double Mt = 0.0, Zt = 0.0, Wt = 0.0, yt = -CUDART_INF;
-      int it_ = -1, et = 0;
-      for (int k = s.k0; k <= s.k1; ++k) {
-        // CTA k keeps this row's piece in slot 0 when the row is the first thing it works on
-        const bool is_first_seg = first_tile_of(p, k) / p.tiles_per_row == s.row;
-        const volatile Piece *q = pieces + (size_t)k * 2 + (is_first_seg ? 0 : 1);
-        const double M2 = q->M, Z2 = q->Z, W2 = q->W, y2 = q->y;
-        const int i2 = q->idx;
-        et |= q->err;
-        merge_stats_d(Mt, Zt, Wt, M2, Z2, W2);
-        merge_best(yt, it_, y2, i2);
-      }
-      finish_row<DT>(p, s.row, ri, Mt, Zt, Wt, yt, it_, et);
+      if (lane == 0) finish_row<DT>(p, s.row, ri, Md, Zd, Wd, yd, id, ed);
     }
   }
 }
@@ -1075,9 +1427,11 @@ cudaError_t launch_rows(RowsParams p, int dtype, int sampler, bool aligned, void
   if (dtype == 0) {
     if (sampler < 0) { E3_DISPATCH(0, -1); }
     if (sampler == 0) { E3_DISPATCH(0, 0); }
+    if (sampler == 1) { E3_DISPATCH(0, 1); }
   } else {
     if (sampler < 0) { E3_DISPATCH(1, -1); }
     if (sampler == 0) { E3_DISPATCH(1, 0); }
+    if (sampler == 1) { E3_DISPATCH(1, 1); }
   }
 #undef E3_DISPATCH
   return cudaErrorInvalidValue;

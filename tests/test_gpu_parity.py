@@ -61,11 +61,12 @@ def _check_sample(e3, logits, temps, seed, counter, row_base=0, sampler=0, name=
 # ----------------------------------------------------------------------------------------------
 # configuration 1: 64 rows (8 prompts x 8 rollouts) x 32,000 fp32, full parity incl. advantages
 # ----------------------------------------------------------------------------------------------
-def test_config1_tiny_sampling_step(e3):
+@pytest.mark.parametrize("sampler", [0, 1])
+def test_config1_tiny_sampling_step(e3, sampler):
     rows, V = 64, 32000
     logits = inputs.zipf_gaussian_logits(rows, V, seed=1, dtype=torch.float32, device=DEV)
     temps = inputs.uniform_temps(rows, seed=2, device=DEV)
-    info = _check_sample(e3, logits, temps, seed=0, counter=0, name="c1")
+    info = _check_sample(e3, logits, temps, seed=0, counter=0, sampler=sampler, name="c1")
     assert info["mismatch_near_tie"] == 0
     sizes = [8] * 8
     rewards = inputs.bernoulli_rewards(sizes, 0.5, seed=3, device=DEV)
@@ -78,13 +79,14 @@ def test_config1_tiny_sampling_step(e3):
         assert abs(float(adv[8 * g:8 * g + 8].sum())) < 1e-4
 
 
+@pytest.mark.parametrize("sampler", [0, 1])
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
-def test_rollout_shape_rows_full_vocab(e3, dtype):
-    """A few dozen rows at V = 151,936: several slices per row, every cluster size in play."""
-    for rows, seed in ((3, 10), (41, 11), (150, 12)):
+def test_rollout_shape_rows_full_vocab(e3, dtype, sampler):
+    """Rows at V = 151,936: rows cut between thread blocks (few rows) and whole rows per block (many rows)."""
+    for rows, seed in ((3, 10), (41, 11), (150, 12), (700, 13)):
         logits = inputs.zipf_gaussian_logits(rows, 151936, seed=seed, dtype=dtype, device=DEV)
         temps = inputs.uniform_temps(rows, seed=seed + 50, device=DEV)
-        _check_sample(e3, logits, temps, seed=5, counter=seed, name=f"rollout{rows}")
+        _check_sample(e3, logits, temps, seed=5, counter=seed, sampler=sampler, name=f"rollout{rows}")
 
 
 # ----------------------------------------------------------------------------------------------
@@ -96,7 +98,9 @@ def test_ragged_vocab_sizes(e3, dtype, V):
     for rows in (1, 2, 149):
         logits = inputs.zipf_gaussian_logits(rows, V, seed=V + rows, dtype=dtype, device=DEV)
         temps = inputs.uniform_temps(rows, seed=V, device=DEV)
-        _check_sample(e3, logits, temps, seed=V, counter=(1 << 33) + rows, row_base=7, name=f"V{V}r{rows}")
+        for sampler in (0, 1):
+            _check_sample(e3, logits, temps, seed=V, counter=(1 << 33) + rows, row_base=7, sampler=sampler,
+                          name=f"V{V}r{rows}s{sampler}")
         targets = inputs.uniform_targets(rows, V, seed=3, device=DEV)
         lp, en = e3.e3_token_logp_entropy(logits, targets, temps=temps)
         rlp, ren, _ = oracle.token_logp_entropy(inputs.to_oracle_array(logits), targets.cpu().numpy(),
@@ -113,11 +117,12 @@ def test_padded_stride_and_unaligned_rows(e3, dtype):
     # stride > V, rows still 16-byte aligned
     view = base[:, :V]
     assert view.stride(0) == V + 24
-    _check_sample(e3, view, temps, seed=1, counter=2, name="padded")
-    # stride that breaks 16-byte row alignment, and a base pointer offset by one element
     odd = inputs.zipf_gaussian_logits(rows, V + 3, seed=79, dtype=dtype, device=DEV)
-    _check_sample(e3, odd[:, :V], temps, seed=1, counter=3, name="oddstride")
-    _check_sample(e3, odd[:, 1:V + 1], temps, seed=1, counter=4, name="offset1")
+    for sampler in (0, 1):
+        _check_sample(e3, view, temps, seed=1, counter=2, sampler=sampler, name="padded")
+        # stride that breaks 16-byte row alignment, and a base pointer offset by one element
+        _check_sample(e3, odd[:, :V], temps, seed=1, counter=3, sampler=sampler, name="oddstride")
+        _check_sample(e3, odd[:, 1:V + 1], temps, seed=1, counter=4, sampler=sampler, name="offset1")
 
 
 def test_empty_batch_is_a_noop(e3):
@@ -150,6 +155,11 @@ def test_special_rows(e3, dtype):
     z[7] = torch.linspace(-2, 2, V)                     # sampled at tau = 0: greedy
     logits = z.to(dtype).to(DEV)
     temps = torch.tensor([0.9, 1.0, 1.0, 0.7, 1.0, 1.0, 1.0, 0.0], dtype=torch.float32, device=DEV)
+    tok1, lp1, en1 = _run_sample(e3, logits, temps, seed=3, counter=9, sampler=1)
+    ref1 = oracle.sample(inputs.to_oracle_array(logits), temps.cpu().numpy(), 3, 9, sampler=1)
+    assert np.array_equal(tok1, ref1.tok)
+    assert_close("ent.s1", en1, ref1.ent, ATOL[dtype])
+    assert_close("logp.s1", lp1, ref1.logp, ATOL[dtype])
     tok, lp, en = _run_sample(e3, logits, temps, seed=3, counter=9)
     ref = oracle.sample(inputs.to_oracle_array(logits), temps.cpu().numpy(), 3, 9)
     assert np.array_equal(tok, ref.tok)
@@ -192,6 +202,7 @@ def test_stress_rows_one_hot_and_flat(e3):
     logits = inputs.onehot_flat_logits(rows, V, seed=20, device=DEV)
     temps = inputs.loguniform_temps(rows, seed=21, device=DEV)
     _check_sample(e3, logits, temps, seed=4, counter=1, name="c5")
+    _check_sample(e3, logits, temps, seed=4, counter=1, sampler=1, name="c5.s1")
     targets = inputs.uniform_targets(rows, V, seed=22, device=DEV)
     lp, en = e3.e3_token_logp_entropy(logits, targets, temps=temps)
     rlp, ren, _ = oracle.token_logp_entropy(logits.cpu().numpy(), targets.cpu().numpy(), temps=temps.cpu().numpy())
@@ -229,7 +240,8 @@ def test_bitwise_reproducible_and_row_base(e3):
     assert np.array_equal(tok.cpu().numpy(), a[0])
 
 
-def test_sampler_distribution_on_device(e3):
+@pytest.mark.parametrize("sampler", [0, 1])
+def test_sampler_distribution_on_device(e3, sampler):
     """Chi-square of 200k device draws (advancing step counter) against softmax(z / tau)."""
     import scipy.special
     import scipy.stats
@@ -239,7 +251,7 @@ def test_sampler_distribution_on_device(e3):
     temps = torch.full((rows,), tau, device=DEV)
     toks = []
     for step in range(100):
-        toks.append(e3.e3_sample(logits, temps, 77, step, want_logp=False, want_ent=False)[0])
+        toks.append(e3.e3_sample(logits, temps, 77, step, sampler=sampler, want_logp=False, want_ent=False)[0])
     toks = torch.cat(toks).cpu().numpy()
     p = scipy.special.softmax(row.cpu().numpy()[0].astype(np.float64) / float(np.float32(tau)))
     counts = np.bincount(toks, minlength=V).astype(np.float64)
