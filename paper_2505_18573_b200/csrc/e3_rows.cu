@@ -12,28 +12,39 @@
 // waits for anybody.  (With a response mask, and when no workspace is given, CTAs take whole
 // rows round-robin instead.)
 //
-// Inside a CTA: one warp issues bulk asynchronous copies (cp.async.bulk, no multicast) of 16 KiB
-// into a 6-stage shared-memory ring guarded by mbarriers; eight warps consume the ring,
-// each thread one 16-entry group per stage (= one coarse Philox call); one warp finishes rows
-// (merges the eight warp states, fp64 epilogue, piece protocol) so that the consumers never
-// stall on it.  Every mbarrier wait is bounded: when a wait runs out the CTA stops waiting
-// altogether, finishes its fixed sequence of steps on whatever data it has and marks its rows
-// invalid.
+// Inside a CTA: one thread issues bulk asynchronous copies (cp.async.bulk, no multicast) of 16 KiB
+// into a 4-stage shared-memory ring guarded by mbarriers; eight warps consume the ring, each
+// thread 64 contiguous bytes per stage (read in a swizzled vector order that is free of bank
+// conflicts); one warp finishes rows (merges the eight warp states, fp64 epilogue, piece protocol)
+// so that the consumers never stall on it.  Every role looks one row ahead for its temperature and
+// mask.  Every mbarrier wait is bounded: when a wait runs out the CTA stops waiting altogether,
+// finishes its fixed sequence of steps on whatever data it has and marks its rows invalid.
 //
-// Numerics.  Each thread keeps (R, Z, W): R the largest logit it has seen, Z = sum 2^t,
-// W = sum 2^t * t with t = z*c - R*c and c = log2(e)/tau.  R only grows, and the sums are
-// rescaled when it does.  States merge associatively; the per-row result is formed in fp64:
+// Numerics.  Each thread keeps a reference logit R and the sums Z = sum 2^t, W = sum 2^t * t with
+// t = z*c - R*c and c = log2(e)/tau, two entries per instruction (packed fp32).  The streaming loop
+// never looks for the maximum: R is taken from the first entries of the row piece and stays until a
+// group sum leaves the safe range, which sends that group through a careful out-of-line form that
+// moves R (and also deals with NaN and infinities).  -inf logits are clamped to a huge negative finite
+// value on the way in, which gives them weight 0 without special cases.  States merge
+// associatively; the per-row result is formed in fp64:
 // H = ln Z - ln2 * W / Z,  ln p_tok = (z_tok*c - M) ln2 - ln Z.
 //
 // Sampler 0 (one Gumbel per vocabulary entry).  u_i has 8 coarse + 32 fine bits.  An entry can
 // only win if its coarse byte is 255 (g_i >= 5.5432) or if z_i/tau exceeds the best score so
-// far minus 5.5432, so the fine bits and the logarithms are evaluated for a fraction of a percent
-// of the entries.  Those candidates are queued per warp, screened with an fp32 upper bound and
-// the survivors evaluated in fp64 with the same expression order as the definition: the token
-// never depends on the gating.
+// far minus 5.5432; the second condition is tested on the group sum of 2^t, which bounds every
+// term from above.  Groups that pass are copied (coarse bytes and logits) into a per-warp queue
+// in shared memory with ballot-compacted positions; when 32 are waiting the warp evaluates them,
+// one per lane: an fp32 upper bound first, the survivors in fp64 with the same expression order
+// as the definition.  The token never depends on the gating.
+//
+// Sampler 1 (one Gumbel per block of 256 entries).  8 (bf16) or 16 (fp32) neighbouring lanes hold
+// one block per step; their sums are added with shuffles, each lane parks one block and all lanes
+// score their parked blocks together.
 #include "e3_rows.cuh"
 
+#include <limits.h>
 #include <math_constants.h>
+#include <string.h>
 
 #include <atomic>
 #include <chrono>
@@ -42,8 +53,11 @@
 namespace e3 {
 namespace {
 
-constexpr int kQueueCap = 192;
-constexpr int kDrainEvery = 4;  // chunks between drains (power of two)
+using u64 = unsigned long long;
+
+constexpr int kQueueCap = 64;   // candidate groups a warp can hold
+constexpr int kDrainAt = 32;    // ... and the fill at which it evaluates them (one per lane)
+constexpr int kQueueHdrBytes = kQueueCap * 4;
 constexpr int kSlots = 4;  // hand-over slots between the consumer warps and the finishing warp
 constexpr uint32_t kSpinLimit = 1u << 23;  // polls before a wait gives up (seconds)
 constexpr float kLog2e = 1.4426950408889634f;
@@ -53,18 +67,41 @@ constexpr double kLn2 = 0.6931471805599453094;
 // with all 40 bits set the largest value is -ln(-ln(1 - 2^-41)) = 28.41903...  Both rounded up.
 constexpr float kGumbelCapCoarse = 5.5433f;
 constexpr float kGumbelCapAll = 28.4192f;
+// A group whose sum of 2^t is above this (or NaN) leaves the streaming form: its reference is stale.
+constexpr float kGroupSumMax = 1.0995116e12f;  // 2^40
+// Logits below this (also -inf) enter the streaming form as this value: weight 2^-huge = 0.
+constexpr uint32_t kFloorBf16x2 = 0xF180F180u;  // -2^100 twice
+constexpr float kFloorF32 = -1.2676506e30f;     // -2^100
 
 enum : int { kErrValue = 1, kErrTimeout = 4 };
 
-struct Piece {  // one partial row state in the workspace (kPieceBytes)
-  double M, Z, W;  // reference (log2 units), sum 2^t, sum 2^t t
+template <int DT>
+struct Fmt {
+  static constexpr int kEsize = DT == 0 ? 4 : 2;
+  static constexpr int kLaneE = kLaneBytes / kEsize;          // entries per thread and stage: 16 fp32 / 32 bf16
+  static constexpr int kG = kLaneE / kGroup;                  // groups per thread and stage: 1 / 2
+  static constexpr int kVG = 4 / kG;                          // 16-byte vectors per group: 4 / 2
+  static constexpr int kChunkE = kStageBytes / kEsize;        // entries per stage: 4,096 / 8,192
+  static constexpr int kEntryBytes = 16 + kGroup * kEsize;    // queue entry: coarse bytes + logits of one group
+  static constexpr int kQueueBytes = kQueueHdrBytes + kQueueCap * kEntryBytes;
+  static constexpr int kLB = 256 / kLaneE;                    // lanes that hold one block of sampler 1: 16 / 8
+};
+
+// One partial row state.  In the workspace it is kPieceWords 64-bit words, each (tag << 32 | payload):
+// the tag depends on the call and on the word, so a reader knows word by word whether what it sees was
+// written by this call (64-bit accesses are single-copy atomic); stale or half-written pieces fail the check.
+struct Piece {
   double y;        // best perturbed score (greedy rows: largest logit)
-  int idx;         // its vocabulary index, -1 = none
+  float M, Z, W;   // reference (log2 units), sum 2^t, sum 2^t t
+  int idx;         // vocabulary index of the best score, -1 = none
+  float zf;        // its logit
   int err;
-  float ty[3];     // sampler 1: the three best block scores (fp32) ...
+  float ty[3];     // sampler 1: the three best block scores (fp32)
   int tb[3];       // ... and their block indices, -1 = none
 };
-static_assert(sizeof(Piece) == kPieceBytes, "piece size");
+constexpr int kPieceWords = 14;
+static_assert(sizeof(Piece) == kPieceWords * 4, "piece payload");
+static_assert(kPieceWords * 8 <= kPieceBytes, "piece size");
 
 struct WarpPartial {
   float M, Z, W;
@@ -73,22 +110,21 @@ struct WarpPartial {
   int err;
   float ty[3];
   int tb[3];
-  int pad;
+  float zf;
 };
 
 struct Smem {
-  unsigned long long full[kStages], empty[kStages];  // ring barriers
-  unsigned long long wfull[kSlots], wfree[kSlots];   // consumer warps -> finishing warp
-  unsigned long long best64;                         // (segment number << 32 | encoded best score) of sampler 0
+  u64 full[kStages], empty[kStages];  // ring barriers
+  u64 wfull[kSlots], wfree[kSlots];   // consumer warps -> finishing warp
+  u64 best64;                         // (segment number << 32 | encoded best score) of sampler 0
   WarpPartial wpart[kSlots][kStreamWarps];
-  int queue[kStreamWarps][kQueueCap];
-  int timeout;                                       // set when a bounded wait ran out
+  int timeout;                        // set when a bounded wait ran out
 };
 
 struct RowInfo {
   float tau, c;
-  bool skip;     // masked out, or invalid temperature: no data is read
-  bool invalid;  // temperature not usable
+  bool masked;   // masked out: the row's logits are not read and nothing is computed
+  bool invalid;  // temperature not usable: the logits still pass through the ring, unused
   bool greedy;
 };
 
@@ -101,13 +137,20 @@ struct Seg {
   int k0, k1;      // CTAs holding the first / last tile of the row (cut rows only)
 };
 
+// Running sums of a consumer thread, two fp32 lanes per register pair.
 struct Acc {
-  float R, nRc, Z0, Z1, W0, W1;
+  float R, nRc;      // reference logit and -R*c; R = -inf, nRc = kNoRef: no reference yet
+  u64 Z2, Wa2, Wb2;  // Z = sum of both halves of Z2, W = sum of the four halves of Wa2, Wb2
+};
+// The same state as plain scalars (careful form).
+struct AccS {
+  float R, nRc, Z, W;
 };
 
 struct Best {
   double y;
   int idx;
+  float zf;     // logit of entry idx
   int enc;      // encoded lower bound of the row's best score known to this thread
   float zthr;   // logit above which an entry may win whatever its coarse byte
   float zthr2;  // logit above which an entry with coarse byte 255 may win
@@ -126,24 +169,58 @@ __device__ __forceinline__ float lg2f(float x) {
   asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
-__device__ __forceinline__ uint32_t max_bf16x2(uint32_t a, uint32_t b) {
-  uint32_t d;
-  asm("max.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+__device__ __forceinline__ u64 pack2(uint32_t lo, uint32_t hi) {
+  u64 d;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "r"(lo), "r"(hi));
   return d;
+}
+__device__ __forceinline__ u64 pack2f(float lo, float hi) { return pack2(__float_as_uint(lo), __float_as_uint(hi)); }
+__device__ __forceinline__ void unpack2(u64 v, float &lo, float &hi) {
+  uint32_t a, b;
+  asm("mov.b64 {%0, %1}, %2;" : "=r"(a), "=r"(b) : "l"(v));
+  lo = __uint_as_float(a);
+  hi = __uint_as_float(b);
+}
+__device__ __forceinline__ float sum2(u64 v) {
+  float a, b;
+  unpack2(v, a, b);
+  return a + b;
+}
+// Packed fp32 arithmetic: both halves of a 64-bit register pair in one instruction.
+__device__ __forceinline__ u64 fma2(u64 a, u64 b, u64 c) {
+  u64 d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ u64 add2(u64 a, u64 b) {
+  u64 d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+// max that keeps NaN (a NaN logit must reach the sums)
+__device__ __forceinline__ uint32_t floor_bf16x2(uint32_t w) {
+  uint32_t d;
+  asm("max.NaN.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(w), "r"(kFloorBf16x2));
+  return d;
+}
+__device__ __forceinline__ uint32_t floor_f32(uint32_t w) {
+  float d;
+  asm("max.NaN.f32 %0, %1, %2;" : "=f"(d) : "f"(__uint_as_float(w)), "f"(kFloorF32));
+  return __float_as_uint(d);
 }
 __device__ __forceinline__ uint32_t smem_addr(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
-__device__ __forceinline__ void mbar_init(unsigned long long *b, int count) {
+__device__ __forceinline__ void mbar_init(u64 *b, int count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(b)), "r"(count) : "memory");
 }
-__device__ __forceinline__ void mbar_arrive(unsigned long long *b) {
+__device__ __forceinline__ void mbar_arrive(u64 *b) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(b)) : "memory");
 }
-__device__ __forceinline__ void mbar_arrive_expect_tx(unsigned long long *b, uint32_t bytes) {
+__device__ __forceinline__ void mbar_arrive_expect_tx(u64 *b, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(b)), "r"(bytes) : "memory");
 }
 // One poll (the hardware may park the thread for a short, implementation-defined time).
-__device__ __forceinline__ bool mbar_try_wait(unsigned long long *b, uint32_t parity) {
+__device__ __forceinline__ bool mbar_try_wait(u64 *b, uint32_t parity) {
   uint32_t ok;
   asm volatile(
       "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
@@ -154,7 +231,7 @@ __device__ __forceinline__ bool mbar_try_wait(unsigned long long *b, uint32_t pa
 }
 // Bounded wait.  After any wait of the CTA has run out, no wait blocks any more.
 // sleep_ns > 0 parks the thread between polls (roles that mostly wait must not eat issue slots).
-__device__ __noinline__ void mbar_wait_slow(unsigned long long *b, uint32_t parity, Smem &sm, unsigned sleep_ns) {
+__device__ __noinline__ void mbar_wait_slow(u64 *b, uint32_t parity, Smem &sm, unsigned sleep_ns) {
   for (uint32_t it = 0; it < kSpinLimit; ++it) {
     if (mbar_try_wait(b, parity)) return;
     if (*reinterpret_cast<volatile int *>(&sm.timeout)) return;
@@ -162,15 +239,15 @@ __device__ __noinline__ void mbar_wait_slow(unsigned long long *b, uint32_t pari
   }
   *reinterpret_cast<volatile int *>(&sm.timeout) = 1;
 }
-__device__ __forceinline__ void mbar_wait(unsigned long long *b, uint32_t parity, Smem &sm, unsigned sleep_ns = 0) {
+__device__ __forceinline__ void mbar_wait(u64 *b, uint32_t parity, Smem &sm, unsigned sleep_ns = 0) {
   if (!mbar_try_wait(b, parity)) mbar_wait_slow(b, parity, sm, sleep_ns);
 }
 // Whole-warp wait with a single polling lane (used by the finishing warp, which mostly waits).
-__device__ __forceinline__ void mbar_wait_warp(unsigned long long *b, uint32_t parity, Smem &sm, int lane) {
-  if (lane == 0) mbar_wait(b, parity, sm, 2000u);
+__device__ __forceinline__ void mbar_wait_warp(u64 *b, uint32_t parity, Smem &sm, int lane) {
+  if (lane == 0) mbar_wait(b, parity, sm, 100u);
   __syncwarp();
 }
-__device__ __forceinline__ void bulk_copy_g2s(void *dst, const void *src, uint32_t bytes, unsigned long long *bar) {
+__device__ __forceinline__ void bulk_copy_g2s(void *dst, const void *src, uint32_t bytes, u64 *bar) {
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
                    smem_addr(dst)),
                "l"(src), "r"(bytes), "r"(smem_addr(bar))
@@ -201,8 +278,15 @@ __device__ __forceinline__ uint32_t pick_word(const uint4 &w, int k) {
 
 // Bit 7 of every byte that equals 0xFF (exact).
 __device__ __forceinline__ uint32_t ff_bytes(uint32_t w) { return w & 0x80808080u & ((w & 0x7F7F7F7Fu) + 0x01010101u); }
-// Non-zero iff some byte equals 0xFF (cheaper; individual bits may over-report).
-__device__ __forceinline__ uint32_t any_ff(uint32_t w) { return (~w - 0x01010101u) & w & 0x80808080u; }
+// Non-zero iff some byte of the four words equals 0xFF (a byte is 0xFF iff its complement is zero; the
+// borrow of the subtraction can only over-report above a byte that really is 0xFF).
+__device__ __forceinline__ uint32_t any_ff4(const uint4 &w) {
+  uint32_t r = (0xFEFEFEFEu - w.x) & w.x;
+  r |= (0xFEFEFEFEu - w.y) & w.y;
+  r |= (0xFEFEFEFEu - w.z) & w.z;
+  r |= (0xFEFEFEFEu - w.w) & w.w;
+  return r & 0x80808080u;
+}
 
 __device__ __forceinline__ int enc_float(float f) {
   int b = __float_as_int(f);
@@ -213,10 +297,10 @@ __device__ __forceinline__ int enc_neg_inf() { return enc_float(-CUDART_INF_F); 
 
 // CTA-wide best score of the segment: 64-bit word (segment number, order-preserving code).
 __device__ __forceinline__ void post_best(Smem &sm, uint32_t seg, int enc) {
-  atomicMax(&sm.best64, ((unsigned long long)seg << 32) | (uint32_t)(enc ^ 0x80000000));
+  atomicMax(&sm.best64, ((u64)seg << 32) | (uint32_t)(enc ^ 0x80000000));
 }
 __device__ __forceinline__ int read_best(Smem &sm, uint32_t seg) {
-  const unsigned long long v = *reinterpret_cast<volatile unsigned long long *>(&sm.best64);
+  const u64 v = *reinterpret_cast<volatile u64 *>(&sm.best64);
   return (uint32_t)(v >> 32) == seg ? (int)((uint32_t)v ^ 0x80000000u) : enc_neg_inf();
 }
 
@@ -229,6 +313,7 @@ __device__ __forceinline__ float load_elem(const char *row, int64_t i) {
   return __uint_as_float((uint32_t)__ldg(reinterpret_cast<const unsigned short *>(row) + i) << 16);
 }
 
+// 16 logits from global memory, entries at or beyond `valid` read as -inf.  Returns the largest.
 template <int DT>
 __device__ __forceinline__ float load_group_guarded(const char *row, int64_t e0, int valid, float (&z)[16]) {
   float gmax = -CUDART_INF_F;
@@ -240,115 +325,146 @@ __device__ __forceinline__ float load_group_guarded(const char *row, int64_t e0,
   return gmax;
 }
 
-// One full group: raw 16-byte words from a pipeline stage, then widening to fp32.
+// 16 logits that lie contiguously in shared memory (plain order).
 template <int DT>
-struct RawGroup {
-  uint4 q[DT == 0 ? 4 : 2];
-};
-
-template <int DT>
-__device__ __forceinline__ void load_raw_smem(const unsigned char *stage, int slot, RawGroup<DT> &r) {
-  constexpr int kQ = DT == 0 ? 4 : 2;
-  const uint4 *p = reinterpret_cast<const uint4 *>(stage) + slot * kQ;
-#pragma unroll
-  for (int i = 0; i < kQ; ++i) r.q[i] = p[i];
-}
-
-// Returns the group's largest logit.
-template <int DT>
-__device__ __forceinline__ float unpack_group(const RawGroup<DT> &r, float (&z)[16]) {
+__device__ __forceinline__ void load_group_smem(const unsigned char *src, float (&z)[16]) {
   if (DT == 0) {
+    const float4 *p = reinterpret_cast<const float4 *>(src);
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
-      z[4 * q + 0] = __uint_as_float(r.q[q].x); z[4 * q + 1] = __uint_as_float(r.q[q].y);
-      z[4 * q + 2] = __uint_as_float(r.q[q].z); z[4 * q + 3] = __uint_as_float(r.q[q].w);
+      const float4 v = p[q];
+      z[4 * q] = v.x; z[4 * q + 1] = v.y; z[4 * q + 2] = v.z; z[4 * q + 3] = v.w;
     }
-    float m[4];
-#pragma unroll
-    for (int q = 0; q < 4; ++q) m[q] = fmaxf(fmaxf(z[4 * q], z[4 * q + 1]), fmaxf(z[4 * q + 2], z[4 * q + 3]));
-    return fmaxf(fmaxf(m[0], m[1]), fmaxf(m[2], m[3]));
   } else {
-    const uint32_t w[8] = {r.q[0].x, r.q[0].y, r.q[0].z, r.q[0].w, r.q[DT == 0 ? 0 : 1].x, r.q[DT == 0 ? 0 : 1].y,
-                           r.q[DT == 0 ? 0 : 1].z, r.q[DT == 0 ? 0 : 1].w};
+    const uint4 *p = reinterpret_cast<const uint4 *>(src);
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      z[2 * j + 0] = __uint_as_float(w[j] << 16);
-      z[2 * j + 1] = __uint_as_float(w[j] & 0xFFFF0000u);
+    for (int q = 0; q < 2; ++q) {
+      const uint4 v = p[q];
+      const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        z[8 * q + 2 * j] = __uint_as_float(w[j] << 16);
+        z[8 * q + 2 * j + 1] = __uint_as_float(w[j] & 0xFFFF0000u);
+      }
     }
-    const uint32_t m = max_bf16x2(max_bf16x2(max_bf16x2(w[0], w[1]), max_bf16x2(w[2], w[3])),
-                                  max_bf16x2(max_bf16x2(w[4], w[5]), max_bf16x2(w[6], w[7])));
-    return fmaxf(__uint_as_float(m << 16), __uint_as_float(m & 0xFFFF0000u));
   }
 }
 
 // ---------------------------------------------------------------------------------------------
-// Online (R, Z, W) accumulation of one group whose largest logit is gmax.
-// CAREFUL also accepts -inf entries (skipped) and flags NaN; the fast form leaves NaN in the
-// sums when it meets either, which sends the thread's groups through the careful form once more.
+// Running sums
 // ---------------------------------------------------------------------------------------------
-// The reference moves to max(R, gmax) before every group.  The fast form does this without a branch
-// (a per-lane branch that is rarely taken is taken by some lane of the warp almost every time):
-// the sums are multiplied by f = 2^(nRc_new - nRc_old), which is 1 when the reference stays.
-// Acc starts with nRc = kNoRef, a huge finite value, so that the first f is 0 and no inf*0 arises.
-constexpr float kNoRef = 1e30f;
+constexpr float kNoRef = 1e30f;  // nRc of a state without reference: the first group always overflows into the careful form
 
-template <bool CAREFUL>
-__device__ __forceinline__ void accumulate(Acc &a, const float (&z)[16], float c, float gmax, int &err) {
-  if (CAREFUL) {
-    if (gmax > a.R) {
-      if (gmax == CUDART_INF_F) {
-        err |= kErrValue;
-        return;
-      }
-      const float nRc = -gmax * c;
-      const float d = nRc - a.nRc;
-      const float f = ex2f(d);
-      if (f == 0.f) {
-        a.Z0 = a.Z1 = a.W0 = a.W1 = 0.f;
-      } else {
-        a.W0 = f * fmaf(d, a.Z0, a.W0);
-        a.W1 = f * fmaf(d, a.Z1, a.W1);
-        a.Z0 *= f;
-        a.Z1 *= f;
-      }
-      a.R = gmax;
-      a.nRc = nRc;
+__device__ __forceinline__ void acc_reset(Acc &a) {
+  a.R = -CUDART_INF_F;
+  a.nRc = kNoRef;
+  a.Z2 = a.Wa2 = a.Wb2 = 0ull;
+}
+__device__ __forceinline__ AccS to_scalar(const Acc &a) {
+  AccS s;
+  s.R = a.R;
+  s.nRc = a.nRc;
+  s.Z = sum2(a.Z2);
+  s.W = sum2(a.Wa2) + sum2(a.Wb2);
+  return s;
+}
+__device__ __forceinline__ void from_scalar(Acc &a, const AccS &s) {
+  a.R = s.R;
+  a.nRc = s.nRc;
+  a.Z2 = pack2f(s.Z, 0.f);
+  a.Wa2 = pack2f(s.W, 0.f);
+  a.Wb2 = 0ull;
+}
+
+// Careful form for one group: accepts any values.  -inf entries carry no weight, NaN and +inf flag the
+// row.  The reference moves up to max(R, ref_floor, largest logit of the group).  Returns the group's
+// sum of 2^t under the reference the state has afterwards.
+__device__ __forceinline__ float careful_accumulate(AccS &a, const float (&z)[16], float c, float ref_floor, int &err) {
+  float gmax = ref_floor;
+#pragma unroll
+  for (int k = 0; k < 16; ++k) {
+    if (z[k] != z[k]) err |= kErrValue;
+    gmax = fmaxf(gmax, z[k]);
+  }
+  if (gmax == CUDART_INF_F) {
+    err |= kErrValue;
+    return 0.f;
+  }
+  if (gmax > a.R) {
+    const float nRc = -gmax * c;
+    if (!(fabsf(nRc) < CUDART_INF_F)) {  // the product left the fp32 range
+      err |= kErrValue;
+      return 0.f;
     }
-  } else {
-    const float R = fmaxf(a.R, gmax);  // +inf or NaN logits end up as NaN in the sums and are sorted out later
-    const float nRc = -R * c;
-    const float d = nRc - a.nRc;       // <= 0
-    const float f = ex2f(d);
-    a.W0 = f * fmaf(d, a.Z0, a.W0);
-    a.W1 = f * fmaf(d, a.Z1, a.W1);
-    a.Z0 *= f;
-    a.Z1 *= f;
-    a.R = R;
+    const float d = nRc - a.nRc;
+    const float f = a.R == -CUDART_INF_F ? 0.f : ex2f(d);
+    if (f == 0.f) {
+      a.Z = a.W = 0.f;
+    } else {
+      a.W = f * fmaf(d, a.Z, a.W);
+      a.Z *= f;
+    }
+    a.R = gmax;
     a.nRc = nRc;
   }
+  float g = 0.f;
 #pragma unroll
-  for (int k = 0; k < 16; k += 2) {
-    if (CAREFUL) {
-      if (z[k] != z[k] || z[k + 1] != z[k + 1]) err |= kErrValue;
-      if (z[k] != -CUDART_INF_F && z[k] == z[k]) {
-        const float t = fmaf(z[k], c, a.nRc), e = ex2f(t);
-        a.Z0 += e;
-        a.W0 = fmaf(e, t, a.W0);
-      }
-      if (z[k + 1] != -CUDART_INF_F && z[k + 1] == z[k + 1]) {
-        const float t = fmaf(z[k + 1], c, a.nRc), e = ex2f(t);
-        a.Z1 += e;
-        a.W1 = fmaf(e, t, a.W1);
-      }
-    } else {
-      const float t0 = fmaf(z[k], c, a.nRc), t1 = fmaf(z[k + 1], c, a.nRc);
-      const float e0 = ex2f(t0), e1 = ex2f(t1);
-      a.Z0 += e0;
-      a.Z1 += e1;
-      a.W0 = fmaf(e0, t0, a.W0);
-      a.W1 = fmaf(e1, t1, a.W1);
+  for (int k = 0; k < 16; ++k) {
+    if (z[k] > -CUDART_INF_F) {  // false for NaN as well
+      const float t = fmaf(z[k], c, a.nRc), e = ex2f(t);
+      g += e;
+      a.W = fmaf(e, t, a.W);
     }
   }
+  a.Z += g;
+  return g;
+}
+
+// Streaming form for one group held in raw 16-byte vectors (any order): adds sum 2^t t to (Wa2, Wb2),
+// returns the packed group sum of 2^t in Zg2 and its scalar value.
+template <int DT>
+__device__ __forceinline__ float hot_group(const uint4 *v, u64 c2, u64 nRc2, u64 &Wa2, u64 &Wb2, u64 &Zg2) {
+  u64 Za = 0ull, Zb = 0ull;
+#pragma unroll
+  for (int q = 0; q < Fmt<DT>::kVG; ++q) {
+    const uint32_t w[4] = {v[q].x, v[q].y, v[q].z, v[q].w};
+    if (DT == 1) {
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const uint32_t x = floor_bf16x2(w[j]);
+        const u64 z2 = pack2(x << 16, x & 0xFFFF0000u);
+        const u64 t2 = fma2(z2, c2, nRc2);
+        float tl, th;
+        unpack2(t2, tl, th);
+        const u64 e2 = pack2f(ex2f(tl), ex2f(th));
+        if (j & 1) {
+          Zb = (q == 0 && j == 1) ? e2 : add2(Zb, e2);
+          Wb2 = fma2(e2, t2, Wb2);
+        } else {
+          Za = (q == 0 && j == 0) ? e2 : add2(Za, e2);
+          Wa2 = fma2(e2, t2, Wa2);
+        }
+      }
+    } else {
+#pragma unroll
+      for (int j = 0; j < 2; ++j) {
+        const u64 z2 = pack2(floor_f32(w[2 * j]), floor_f32(w[2 * j + 1]));
+        const u64 t2 = fma2(z2, c2, nRc2);
+        float tl, th;
+        unpack2(t2, tl, th);
+        const u64 e2 = pack2f(ex2f(tl), ex2f(th));
+        if (j & 1) {
+          Zb = (q == 0) ? e2 : add2(Zb, e2);
+          Wb2 = fma2(e2, t2, Wb2);
+        } else {
+          Za = (q == 0) ? e2 : add2(Za, e2);
+          Wa2 = fma2(e2, t2, Wa2);
+        }
+      }
+    }
+  }
+  Zg2 = add2(Za, Zb);
+  return sum2(Zg2);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -362,6 +478,17 @@ __device__ __forceinline__ void set_gate(Best &b, int enc, float tau) {
   b.zthr = t1 - fabsf(t1) * 1e-6f - 1e-30f;
   b.zthr2 = t2 - fabsf(t2) * 1e-6f - 1e-30f;
   if (enc == enc_neg_inf()) b.zthr = b.zthr2 = -CUDART_INF_F;
+}
+
+// The gate of the streaming loop: an entry whose coarse byte is below 255 can only win if
+// 2^t_i > 2^((B - 5.5433) log2 e - R c); the group sum of 2^t bounds every term from above.  The slack
+// covers the fp32 roundings of t_i, of the threshold and of the approximate 2^x.
+__device__ __forceinline__ float gate_threshold(int enc, float nRc) {
+  if (enc == enc_neg_inf()) return 0.f;
+  const float B = dec_float(enc);
+  const float a = (B - kGumbelCapCoarse) * kLog2e;
+  const float t = a + nRc - (1e-3f + (fabsf(a) + fabsf(nRc)) * 4e-7f);
+  return ex2f(t);  // 0 when far below the range (every group with weight passes), +inf when far above
 }
 
 struct EvalCtx {
@@ -399,6 +526,7 @@ __device__ __noinline__ void eval_element(const EvalCtx &x, int i, uint32_t cbyt
   if (y > b.y || (y == b.y && i < b.idx)) {
     b.y = y;
     b.idx = i;
+    b.zf = zf;
     const int enc = enc_float(__double2float_rd(y));
     if (enc > b.enc) {
       set_gate(b, enc, x.tau);
@@ -407,214 +535,69 @@ __device__ __noinline__ void eval_element(const EvalCtx &x, int i, uint32_t cbyt
   }
 }
 
-// A queue entry names one 16-entry group: (group index << 5) | flags.  Flag bits 0-3: the coarse
-// bytes of word 0-3 contain 0xFF (may over-report); bit 4: some logit of the group is above the gate.
-// Each warp owns a queue; its fill count lives in a warp-uniform register, positions come from a
-// ballot, so queueing costs no atomics.  A chunk adds at most 32 entries per group slot, and the
-// queue is drained as soon as it holds 32, so kQueueCap >= 31 + 32 * (groups per thread) suffices.
+// A queue entry holds one group: 16 coarse bytes, then its 16 logits in vocabulary order.  Its header
+// word is the index of the group's first entry, with bit 0 set when the group passed the sum gate.
 template <int DT>
-__device__ __noinline__ void eval_entry(const EvalCtx &x, int entry, Best &b, Smem &sm, bool aligned) {
-  const int base = (entry >> 5) << 4;
-  // all 16 logits of the group first (independent loads, one memory latency), then the coarse bytes
-  float z[16];
-  if (aligned && base + 16 <= x.V) {
-    if (DT == 0) {
-      const float4 *p = reinterpret_cast<const float4 *>(x.row) + (base >> 2);
-#pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        const float4 v = __ldg(p + q);
-        z[4 * q] = v.x; z[4 * q + 1] = v.y; z[4 * q + 2] = v.z; z[4 * q + 3] = v.w;
-      }
-    } else {
-      const uint4 *p = reinterpret_cast<const uint4 *>(x.row) + (base >> 3);
-#pragma unroll
-      for (int q = 0; q < 2; ++q) {
-        const uint4 v = __ldg(p + q);
-        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          z[8 * q + 2 * j] = __uint_as_float(w[j] << 16);
-          z[8 * q + 2 * j + 1] = __uint_as_float(w[j] & 0xFFFF0000u);
-        }
-      }
-    }
-  } else {
-    load_group_guarded<DT>(x.row, base, x.V - base, z);
-  }
-  const uint4 cw = philox(x.rk, (uint32_t)base >> 4, x.grow, x.ctr_lo, x.ctr_hi8 | 0u);
-  const bool over = (entry & 16) != 0;
-  // which of the 16 entries need a look (no calls in this loop), then one pass per set bit
+__device__ __forceinline__ float entry_logit(const unsigned char *entry, int k) {
+  if (DT == 0) return *reinterpret_cast<const float *>(entry + 16 + 4 * k);
+  return __uint_as_float((uint32_t)(*reinterpret_cast<const unsigned short *>(entry + 16 + 2 * k)) << 16);
+}
+
+template <int DT>
+__device__ __forceinline__ void eval_entry(const EvalCtx &x, const unsigned char *entry, int hdr, Best &b, Smem &sm) {
+  const int base = hdr & ~15;
+  const uint4 cw = *reinterpret_cast<const uint4 *>(entry);
   uint32_t todo = 0;
+  {
+    const uint32_t w[4] = {cw.x, cw.y, cw.z, cw.w};
 #pragma unroll
-  for (int k = 0; k < 16; ++k) {
-    const uint32_t cbyte = (pick_word(cw, k >> 2) >> (8 * (k & 3))) & 0xFFu;
-    todo |= ((cbyte == 255u || (over && z[k] > b.zthr)) ? 1u : 0u) << k;
+    for (int q = 0; q < 4; ++q) {
+      const uint32_t m = ff_bytes(w[q]);
+      todo |= (((m >> 7) & 1u) | ((m >> 14) & 2u) | ((m >> 21) & 4u) | ((m >> 28) & 8u)) << (4 * q);
+    }
+  }
+  if (hdr & 1) {
+#pragma unroll 1
+    for (int k = 0; k < 16; ++k)
+      if (entry_logit<DT>(entry, k) > b.zthr) todo |= 1u << k;
   }
   while (todo) {
     const int k = __ffs(todo) - 1;
     todo &= todo - 1;
+    eval_element(x, base + k, entry[k], entry_logit<DT>(entry, k), b, sm);
+  }
+}
+
+// Evaluates the warp's queued groups, one per lane and round.
+template <int DT>
+__device__ __noinline__ void drain_queue(const EvalCtx &x, Best &b, Smem &sm, const unsigned char *queue, int qn) {
+  const int lane = threadIdx.x & 31;
+  __syncwarp();
+  const int *hdr = reinterpret_cast<const int *>(queue);
+  for (int e = lane; e < qn; e += 32)
+    eval_entry<DT>(x, queue + kQueueHdrBytes + e * Fmt<DT>::kEntryBytes, hdr[e], b, sm);
+  __syncwarp();
+}
+
+// Direct evaluation of one group held as floats (paths that do not stream from the ring).
+__device__ __forceinline__ void eval_group_direct(const EvalCtx &x, const float (&z)[16], int e0, int valid, Best &b,
+                                                  Smem &sm) {
+  if (valid <= 0) return;
+  const uint4 cw = philox(x.rk, (uint32_t)e0 >> 4, x.grow, x.ctr_lo, x.ctr_hi8 | 0u);
+#pragma unroll 1
+  for (int k = 0; k < valid; ++k) {
     const uint32_t cbyte = (pick_word(cw, k >> 2) >> (8 * (k & 3))) & 0xFFu;
-    eval_element(x, base + k, cbyte, z[k], b, sm);  // padding beyond the row is -inf and drops out there
+    if (cbyte == 255u || z[k] > b.zthr) eval_element(x, e0 + k, cbyte, z[k], b, sm);
   }
-}
-
-template <int DT>
-__device__ __forceinline__ void drain_queue(const EvalCtx &x, Best &b, Smem &sm, int warp, int lane, int &qn,
-                                            bool aligned) {
-  __syncwarp();
-  for (int e = lane; e < qn; e += 32) eval_entry<DT>(x, sm.queue[warp][e], b, sm, aligned);
-  __syncwarp();
-  qn = 0;
-}
-
-// First step of a segment (warp-uniform): a valid lower bound of the row's best score from the coarse
-// byte of each lane's largest entry alone: u >= (c + 2^-33)/256  =>  g >= -ln(ln 256 - ln(c + 2^-33)).
-__device__ __forceinline__ void seed_gate(const EvalCtx &x, const float (&z)[16], float gmax, bool have,
-                                          const uint4 &cb, Best &b, Smem &sm) {
-  float ylo = -CUDART_INF_F;
-  if (have && gmax > -CUDART_INF_F && gmax < CUDART_INF_F) {
-    uint32_t cbyte = 0;
-#pragma unroll
-    for (int k = 15; k >= 0; --k)
-      if (z[k] == gmax) cbyte = (pick_word(cb, k >> 2) >> (8 * (k & 3))) & 0xFFu;
-    const float neg_ln_u = (8.0f - lg2f((float)cbyte + 0x1p-33f)) * kLn2f;
-    const float glo = -lg2f(neg_ln_u) * kLn2f;
-    const float sf = gmax / x.tau;
-    ylo = sf - fabsf(sf) * 2e-6f + glo - 2e-3f;
-  }
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) ylo = fmaxf(ylo, __shfl_xor_sync(0xffffffffu, ylo, o));
-  int enc = enc_float(ylo);
-  if ((threadIdx.x & 31) == 0 && enc > enc_neg_inf()) post_best(sm, x.seg, enc);
-  const int cta = read_best(sm, x.seg);
-  enc = enc > cta ? enc : cta;
-  if (enc > b.enc) set_gate(b, enc, x.tau);
-}
-
-// Gate and queue for one group (sampler 0).  qn is the warp's queue fill (warp-uniform).
-__device__ __forceinline__ void sample_group(const EvalCtx &x, float gmax, bool have, int e0, const uint4 &cb, Best &b,
-                                             Smem &sm, int warp, int lane, int &qn) {
-  const uint32_t a0 = any_ff(cb.x), a1 = any_ff(cb.y), a2 = any_ff(cb.z), a3 = any_ff(cb.w);
-  const bool over = have && gmax > b.zthr;
-  const bool flag = (a0 | a1 | a2 | a3) != 0u || over;
-  const uint32_t ballot = __ballot_sync(0xffffffffu, flag);
-  if (ballot != 0u) {
-    if (flag) {
-      const int entry = ((e0 >> 4) << 5) | (over ? 16 : 0) | (a0 ? 1 : 0) | (a1 ? 2 : 0) | (a2 ? 4 : 0) | (a3 ? 8 : 0);
-      sm.queue[warp][qn + __popc(ballot & ((1u << lane) - 1u))] = entry;
-    }
-    qn += __popc(ballot);
-  }
-}
-
-// A consumer thread's running state for the segment it is working on.
-struct LaneState {
-  Acc acc;
-  Best best;
-  int err;
-  int qn;  // fill of the warp's candidate queue (warp-uniform)
-};
-
-// The common case, kept small so that the streaming loop stays in the instruction cache: a full group
-// read from the pipeline stage, finite logits assumed, gate already seeded.
-template <int DT, int SAMPLER>
-__device__ __forceinline__ void hot_group(const EvalCtx &x, const unsigned char *stage, int slot, int e0, float c,
-                                          bool have, Acc &acc, Best &best, int &err, int &qn, Smem &sm, int warp,
-                                          int lane) {
-  float gmax = -CUDART_INF_F;
-  if (have) {
-    RawGroup<DT> raw;
-    load_raw_smem<DT>(stage, slot, raw);
-    float z[16];
-    gmax = unpack_group<DT>(raw, z);
-    accumulate<false>(acc, z, c, gmax, err);
-  }
-  if (SAMPLER == 0) {
-    uint4 cb = make_uint4(0, 0, 0, 0);
-    if (have) cb = philox(x.rk, (uint32_t)e0 >> 4, x.grow, x.ctr_lo, x.ctr_hi8 | 0u);
-    sample_group(x, gmax, have, e0, cb, best, sm, warp, lane, qn);
-  }
-}
-
-// Everything else: the first chunk of a segment (seeds the gate), ragged chunks, rows that do not end on
-// a group boundary, greedy rows, rows that cannot use the ring.  One call handles the thread's group
-// `slot` of the chunk that starts at entry `cs`.
-template <int DT, int SAMPLER>
-__device__ __noinline__ void slow_group(const EvalCtx &x, const unsigned char *stage, int slot, int cs, int e_hi,
-                                        float c, bool greedy, bool seed, LaneState &st, Smem &sm) {
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int e0 = cs + slot * kGroup;
-  const bool have = e0 < e_hi;
-  const bool full = e0 + kGroup <= x.V;
-  float z[16];
-  float gmax = -CUDART_INF_F;
-  if (have && full && stage != nullptr) {
-    RawGroup<DT> raw;
-    load_raw_smem<DT>(stage, slot, raw);
-    gmax = unpack_group<DT>(raw, z);
-  } else if (have) {
-    gmax = load_group_guarded<DT>(x.row, e0, full ? 16 : x.V - e0, z);
-  } else {
-#pragma unroll
-    for (int k = 0; k < 16; ++k) z[k] = -CUDART_INF_F;
-  }
-  if (greedy) {
-    if (have) {
-      int kk = -1;
-#pragma unroll
-      for (int k = 15; k >= 0; --k) {
-        if (z[k] != z[k] || z[k] == CUDART_INF_F) st.err |= kErrValue;
-        if (z[k] == gmax) kk = k;
-      }
-      if (kk >= 0 && gmax > -CUDART_INF_F && (double)gmax > st.best.y) {
-        st.best.y = (double)gmax;
-        st.best.idx = e0 + kk;
-      }
-    }
-    return;
-  }
-  if (have) {
-    if (full && stage != nullptr)
-      accumulate<false>(st.acc, z, c, gmax, st.err);
-    else
-      accumulate<true>(st.acc, z, c, gmax, st.err);
-  }
-  if (SAMPLER == 0) {
-    uint4 cb = make_uint4(0, 0, 0, 0);
-    if (have) cb = philox(x.rk, (uint32_t)e0 >> 4, x.grow, x.ctr_lo, x.ctr_hi8 | 0u);
-    if (seed) seed_gate(x, z, gmax, have, cb, st.best, sm);
-    sample_group(x, gmax, have, e0, cb, st.best, sm, warp, lane, st.qn);
-  }
-}
-
-// Seeds the gate of sampler 0 from the thread's first group of a segment (full groups read from the
-// stage; other lanes contribute nothing).  Called once per segment, before the streaming loop.
-template <int DT>
-__device__ __noinline__ void seed_from_stage(const EvalCtx &x, const unsigned char *stage, int slot, int e0,
-                                             bool usable, Best &b, Smem &sm) {
-  float z[16];
-  float gmax = -CUDART_INF_F;
-  uint4 cb = make_uint4(0, 0, 0, 0);
-  if (usable) {
-    RawGroup<DT> raw;
-    load_raw_smem<DT>(stage, slot, raw);
-    gmax = unpack_group<DT>(raw, z);
-    cb = philox(x.rk, (uint32_t)e0 >> 4, x.grow, x.ctr_lo, x.ctr_hi8 | 0u);
-  } else {
-#pragma unroll
-    for (int k = 0; k < 16; ++k) z[k] = -CUDART_INF_F;
-  }
-  seed_gate(x, z, gmax, usable, cb, b, sm);
 }
 
 // ---------------------------------------------------------------------------------------------
 // Sampler 1: one Gumbel per block of 256 consecutive entries, applied to the block's log-sum-exp.
-// A block is 16 consecutive groups, i.e. one half-warp in one step.  All lanes of a warp keep the
-// same reference (the warp-wide largest logit so far), so that the 16 group sums of a block add up
-// directly.  Each half-warp parks one block sum per step in one of its lanes; every 16 steps all
-// lanes turn their parked block into a score Y_b = L_b + g_b (one Philox call and three MUFU each)
-// and keep the three best (fp32).  The finishing warp settles near-ties in fp64 and draws the
-// token inside the winning block by inverse CDF.
+// All lanes of a warp keep the same reference, so that the lane sums of a block add up directly.
+// kLB neighbouring lanes hold one block per step; every lane parks one block sum per kLB steps and
+// then all lanes turn their parked block into a score Y_b = L_b + g_b (one Philox call and three
+// MUFU each) and keep the three best (fp32).  The finishing warp settles near-ties in fp64 and
+// draws the token inside the winning block by inverse CDF.
 // ---------------------------------------------------------------------------------------------
 struct Top3 {
   float y[3];
@@ -638,10 +621,6 @@ __device__ __forceinline__ void top3_insert(Top3 &t, float y, int b) {
     t.y[2] = y; t.b[2] = b;
   }
 }
-__device__ __forceinline__ void top3_merge(Top3 &t, const Top3 &o) {
-#pragma unroll
-  for (int i = 0; i < 3; ++i) top3_insert(t, o.y[i], o.b[i]);
-}
 
 struct BlockState {
   Top3 top;
@@ -655,8 +634,9 @@ __device__ __forceinline__ void block_state_reset(BlockState &bs) {
 }
 
 // fp32 Gumbel variate of block b: u = (x + 1/2) 2^-32, g = -ln(-ln u)
-__device__ __forceinline__ float block_gumbel_f32(const EvalCtx &x, int b) {
-  const uint4 w = philox(x.rk, (uint32_t)b >> 2, x.grow, x.ctr_lo, x.ctr_hi8 | 2u);
+__device__ __forceinline__ float block_gumbel_f32(const uint32_t *rk, uint32_t grow, uint32_t ctr_lo, uint32_t ctr_hi8,
+                                                  int b) {
+  const uint4 w = philox(rk, (uint32_t)b >> 2, grow, ctr_lo, ctr_hi8 | 2u);
   const uint32_t xw = pick_word(w, b & 3);
   float a;  // -ln u
   if (xw >= 0xFE000000u) {
@@ -668,110 +648,206 @@ __device__ __forceinline__ float block_gumbel_f32(const EvalCtx &x, int b) {
   return -lg2f(a) * kLn2f;
 }
 
-__device__ __forceinline__ void block_flush(const EvalCtx &x, BlockState &bs) {
+__device__ __noinline__ void block_flush(const uint32_t *rk, uint32_t grow, uint32_t ctr_lo, uint32_t ctr_hi8,
+                                         BlockState &bs) {
   if (bs.b >= 0 && bs.S > 0.f) {
     const float L = (lg2f(bs.S) - bs.ref) * kLn2f;  // ln sum_i exp(s_i) over the block
-    top3_insert(bs.top, L + block_gumbel_f32(x, bs.b), bs.b);
+    top3_insert(bs.top, L + block_gumbel_f32(rk, grow, ctr_lo, ctr_hi8, bs.b), bs.b);
   }
   bs.S = 0.f;
   bs.b = -1;
 }
 
-// One step of a warp: every lane brings (at most) one group.  CAREFUL lanes skip -inf / NaN entries.
-template <bool CAREFUL>
-__device__ __forceinline__ void block_step(const EvalCtx &x, const float (&z)[16], float gmax, bool have, int e0,
-                                           float c, Acc &a, BlockState &bs, int &err, int lane) {
-  if (CAREFUL && have && gmax == CUDART_INF_F) err |= kErrValue;
-  const int mw = __reduce_max_sync(0xffffffffu, enc_float(have ? gmax : -CUDART_INF_F));
-  if (mw != enc_neg_inf()) {  // warp-uniform
-    const float R = fmaxf(a.R, dec_float(mw));
-    const float nRc = -R * c;
-    const float d = nRc - a.nRc;
-    const float f = ex2f(d);
-    a.W0 = f * fmaf(d, a.Z0, a.W0);
-    a.W1 = f * fmaf(d, a.Z1, a.W1);
-    a.Z0 *= f;
-    a.Z1 *= f;
-    a.R = R;
-    a.nRc = nRc;
-    float g0 = 0.f, g1 = 0.f;
-    if (have) {
+// One step of a warp: every lane brings the sum of 2^t over its entries of this step (all lanes under
+// the reference nRc), which lie in block `b`.
+template <int DT>
+__device__ __forceinline__ void block_step(float zlane, int b, float nRc, const uint32_t *rk, uint32_t grow,
+                                           uint32_t ctr_lo, uint32_t ctr_hi8, BlockState &bs, int lane) {
+  constexpr int kLB = Fmt<DT>::kLB;
+  float sb = zlane;
 #pragma unroll
-      for (int k = 0; k < 16; k += 2) {
-        if (CAREFUL) {
-          if (z[k] != z[k] || z[k + 1] != z[k + 1]) err |= kErrValue;
-          if (z[k] != -CUDART_INF_F && z[k] == z[k]) {
-            const float t = fmaf(z[k], c, nRc), e = ex2f(t);
-            g0 += e;
-            a.W0 = fmaf(e, t, a.W0);
-          }
-          if (z[k + 1] != -CUDART_INF_F && z[k + 1] == z[k + 1]) {
-            const float t = fmaf(z[k + 1], c, nRc), e = ex2f(t);
-            g1 += e;
-            a.W1 = fmaf(e, t, a.W1);
-          }
-        } else {
-          const float t0 = fmaf(z[k], c, nRc), t1 = fmaf(z[k + 1], c, nRc);
-          const float e0_ = ex2f(t0), e1_ = ex2f(t1);
-          g0 += e0_;
-          g1 += e1_;
-          a.W0 = fmaf(e0_, t0, a.W0);
-          a.W1 = fmaf(e1_, t1, a.W1);
-        }
-      }
-      a.Z0 += g0;
-      a.Z1 += g1;
-    }
-    float sb = g0 + g1;
-#pragma unroll
-    for (int o = 1; o < 16; o <<= 1) sb += __shfl_xor_sync(0xffffffffu, sb, o);
-    if ((bs.it & 15) == (lane & 15)) {
-      bs.S = sb;
-      bs.ref = nRc;
-      bs.b = e0 >> 8;
-    }
+  for (int o = 1; o < kLB; o <<= 1) sb += __shfl_xor_sync(0xffffffffu, sb, o);
+  if ((bs.it & (kLB - 1)) == (lane & (kLB - 1))) {
+    bs.S = sb;
+    bs.ref = nRc;
+    bs.b = b;
   }
   ++bs.it;
-  if ((bs.it & 15) == 0) block_flush(x, bs);
+  if ((bs.it & (kLB - 1)) == 0) {
+    BlockState t = bs;
+    block_flush(rk, grow, ctr_lo, ctr_hi8, t);
+    bs = t;
+  }
 }
 
-template <int DT>
-__device__ __forceinline__ void hot_group_blocks(const EvalCtx &x, const unsigned char *stage, int slot, int e0,
-                                                 float c, Acc &acc, BlockState &bs, int &err, int lane) {
-  RawGroup<DT> raw;
-  load_raw_smem<DT>(stage, slot, raw);
-  float z[16];
-  const float gmax = unpack_group<DT>(raw, z);
-  block_step<false>(x, z, gmax, true, e0, c, acc, bs, err, lane);
-}
-
-struct LaneStateBlocks {
+// ---------------------------------------------------------------------------------------------
+// Out-of-line forms of one consumer step
+// ---------------------------------------------------------------------------------------------
+struct StepIO {
   Acc acc;
-  BlockState bs;
+  float Zg[2];   // per group of the thread (vocabulary order): sum of 2^t under the final reference
+  float Zextra;  // a sum formed before this call, to be carried to the final reference
   int err;
 };
 
-// Out-of-line form: ragged chunks, the row's partial last group, rows that cannot use the ring.
+// Redo of the thread's groups of one stage in the careful form (a group sum left the safe range).
+// `have` bit g: group g of the thread is part of the row piece.  UNIFORM: all lanes of the warp are
+// here and must end with one common reference.
+template <int DT, bool UNIFORM>
+__device__ __noinline__ void redo_step(StepIO &io, const unsigned char *lane_data, int have, float c) {
+  constexpr int kG = Fmt<DT>::kG;
+  AccS a = to_scalar(io.acc);
+  const float nRc_old = a.nRc;
+  float z[kG][16];
+  float gm = -CUDART_INF_F;
+#pragma unroll
+  for (int g = 0; g < kG; ++g) {
+    if (have & (1 << g)) {
+      load_group_smem<DT>(lane_data + g * kGroup * Fmt<DT>::kEsize, z[g]);
+#pragma unroll
+      for (int k = 0; k < 16; ++k) gm = fmaxf(gm, z[g][k]);
+    } else {
+#pragma unroll
+      for (int k = 0; k < 16; ++k) z[g][k] = -CUDART_INF_F;
+    }
+  }
+  float ref_floor = -CUDART_INF_F;
+  if (UNIFORM) {
+    if (gm == CUDART_INF_F) gm = -CUDART_INF_F;  // flagged below; must not become the reference
+    ref_floor = dec_float(__reduce_max_sync(0xffffffffu, enc_float(gm)));
+  }
+  // settle the reference first, so that all group sums of this call refer to the same one
+  float top = ref_floor;
+#pragma unroll
+  for (int g = 0; g < kG; ++g)
+#pragma unroll
+    for (int k = 0; k < 16; ++k) top = fmaxf(top, z[g][k]);
+  if (top == CUDART_INF_F) top = ref_floor;
+#pragma unroll
+  for (int g = 0; g < kG; ++g) io.Zg[g] = careful_accumulate(a, z[g], c, top, io.err);
+  if (a.nRc != nRc_old) io.Zextra = nRc_old == kNoRef ? 0.f : io.Zextra * ex2f(a.nRc - nRc_old);
+  from_scalar(io.acc, a);
+}
+
+struct SlowIO {
+  Acc acc;
+  Best best;
+  float zsum;  // sum of 2^t over the entries handled by this call, under the final reference
+  int err;
+};
+
+// Up to kG groups of the thread read from global memory with guards: entries [e0, e_hi) of the row, at
+// most kLaneE of them.  Used for the last, partial group of a row, for rows that cannot use the ring
+// and for whatever else does not fit the streaming form.  SAMPLER 0 evaluates candidates directly.
+template <int DT, int SAMPLER, bool UNIFORM>
+__device__ __noinline__ void slow_groups(SlowIO &io, const EvalCtx &x, int e0, int e_hi, float c, Smem &sm) {
+  constexpr int kG = Fmt<DT>::kG;
+  AccS a = to_scalar(io.acc);
+  float z[kG][16];
+  int valid[kG];
+  float gm = -CUDART_INF_F;
+#pragma unroll
+  for (int g = 0; g < kG; ++g) {
+    const int g0 = e0 + g * kGroup;
+    valid[g] = e_hi - g0 < 0 ? 0 : (e_hi - g0 > kGroup ? kGroup : e_hi - g0);
+    if (valid[g] > 0) {
+      gm = fmaxf(gm, load_group_guarded<DT>(x.row, g0, valid[g], z[g]));
+    } else {
+#pragma unroll
+      for (int k = 0; k < 16; ++k) z[g][k] = -CUDART_INF_F;
+    }
+  }
+  float top = gm;
+  if (UNIFORM) {
+    if (gm == CUDART_INF_F) gm = -CUDART_INF_F;
+    top = dec_float(__reduce_max_sync(0xffffffffu, enc_float(gm)));
+  }
+  if (top == CUDART_INF_F) top = -CUDART_INF_F;
+  float zs = 0.f;
+#pragma unroll
+  for (int g = 0; g < kG; ++g) {
+    if (valid[g] > 0 || UNIFORM) zs += careful_accumulate(a, z[g], c, top, io.err);
+    if (SAMPLER == 0) eval_group_direct(x, z[g], e0 + g * kGroup, valid[g], io.best, sm);
+  }
+  io.zsum = zs;
+  from_scalar(io.acc, a);
+}
+
+// Greedy rows (tau = 0): largest logit, lowest index; NaN and +inf flag the row.  Full groups below
+// `lim` are read from the thread's 64 bytes of the pipeline stage (when there is one), the rest from
+// global memory with guards.
 template <int DT>
-__device__ __noinline__ void slow_group_blocks(const EvalCtx &x, const unsigned char *stage, int slot, int cs,
-                                               int e_hi, float c, LaneStateBlocks &st) {
-  const int lane = threadIdx.x & 31;
-  const int e0 = cs + slot * kGroup;
-  const bool have = e0 < e_hi;
-  const bool full = e0 + kGroup <= x.V;
+__device__ __noinline__ void greedy_groups(SlowIO &io, const char *row, const unsigned char *lane_data, int e0, int lim,
+                                           int e_hi) {
+  constexpr int kG = Fmt<DT>::kG;
+#pragma unroll 1
+  for (int g = 0; g < kG; ++g) {
+    const int g0 = e0 + g * kGroup;
+    const int valid = e_hi - g0 < 0 ? 0 : (e_hi - g0 > kGroup ? kGroup : e_hi - g0);
+    if (valid <= 0) continue;
+    float z[16];
+    float gmax = -CUDART_INF_F;
+    if (lane_data != nullptr && g0 + kGroup <= lim) {
+      load_group_smem<DT>(lane_data + g * kGroup * Fmt<DT>::kEsize, z);
+#pragma unroll
+      for (int k = 0; k < 16; ++k) gmax = fmaxf(gmax, z[k]);
+    } else {
+      gmax = load_group_guarded<DT>(row, g0, valid, z);
+    }
+    int kk = -1;
+#pragma unroll
+    for (int k = 15; k >= 0; --k) {
+      if (z[k] != z[k] || z[k] == CUDART_INF_F) io.err |= kErrValue;
+      if (z[k] == gmax) kk = k;
+    }
+    if (kk >= 0 && gmax > -CUDART_INF_F && (double)gmax > io.best.y) {
+      io.best.y = (double)gmax;
+      io.best.idx = g0 + kk;
+      io.best.zf = gmax;
+    }
+  }
+}
+
+struct SeedIO {
+  float R0;  // warp-wide reference, -inf = none found
+  Best best;
+};
+
+// First stage of a row piece: a common reference for the warp from each lane's first group, and for
+// sampler 0 a valid lower bound of the piece's best score from the coarse byte of each lane's largest
+// entry alone: u >= (c + 2^-33)/256  =>  g >= -ln(ln 256 - ln(c + 2^-33)).
+template <int DT, int SAMPLER>
+__device__ __noinline__ void seed_piece(SeedIO &io, const EvalCtx &x, const unsigned char *lane_data, int e_lane,
+                                        int lim, Smem &sm) {
+  const bool have = e_lane + kGroup <= lim;
   float z[16];
   float gmax = -CUDART_INF_F;
-  if (have && full && stage != nullptr) {
-    RawGroup<DT> raw;
-    load_raw_smem<DT>(stage, slot, raw);
-    gmax = unpack_group<DT>(raw, z);
-  } else if (have) {
-    gmax = load_group_guarded<DT>(x.row, e0, full ? 16 : x.V - e0, z);
-  } else {
+  if (have) {
+    load_group_smem<DT>(lane_data, z);
 #pragma unroll
-    for (int k = 0; k < 16; ++k) z[k] = -CUDART_INF_F;
+    for (int k = 0; k < 16; ++k) gmax = fmaxf(gmax, z[k]);
   }
-  block_step<true>(x, z, gmax, have, e0, c, st.acc, st.bs, st.err, lane);
+  const bool usable = have && gmax > -CUDART_INF_F && gmax < CUDART_INF_F;
+  io.R0 = dec_float(__reduce_max_sync(0xffffffffu, enc_float(usable ? gmax : -CUDART_INF_F)));
+  if (SAMPLER == 0) {
+    float ylo = -CUDART_INF_F;
+    if (usable) {
+      const uint4 cb = philox(x.rk, (uint32_t)e_lane >> 4, x.grow, x.ctr_lo, x.ctr_hi8 | 0u);
+      uint32_t cbyte = 0;
+#pragma unroll
+      for (int k = 15; k >= 0; --k)
+        if (z[k] == gmax) cbyte = (pick_word(cb, k >> 2) >> (8 * (k & 3))) & 0xFFu;
+      const float neg_ln_u = (8.0f - lg2f((float)cbyte + 0x1p-33f)) * kLn2f;
+      const float glo = -lg2f(neg_ln_u) * kLn2f;
+      const float sf = gmax / x.tau;
+      ylo = sf - fabsf(sf) * 2e-6f + glo - 2e-3f;
+    }
+    int enc = __reduce_max_sync(0xffffffffu, enc_float(ylo));
+    if ((threadIdx.x & 31) == 0 && enc > enc_neg_inf()) post_best(sm, x.seg, enc);
+    const int cta = read_best(sm, x.seg);
+    enc = enc > cta ? enc : cta;
+    if (enc > io.best.enc) set_gate(io.best, enc, x.tau);
+  }
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -791,36 +867,125 @@ __device__ __forceinline__ void merge_stats_f(float &M, float &Z, float &W, floa
   M = Mn;
 }
 
-__device__ __forceinline__ void merge_stats_d(double &M, double &Z, double &W, double M2, double Z2, double W2) {
-  if (Z2 == 0.0) return;
-  if (Z == 0.0) {
-    M = M2; Z = Z2; W = W2;
-    return;
-  }
-  const double Mn = fmax(M, M2);
-  const double d1 = M - Mn, d2 = M2 - Mn;
-  const double a = exp2(d1), b = exp2(d2);
-  W = a * (W + d1 * Z) + b * (W2 + d2 * Z2);
-  Z = a * Z + b * Z2;
-  M = Mn;
-}
-
-__device__ __forceinline__ void merge_best(double &y, int &idx, double y2, int idx2) {
+__device__ __forceinline__ void merge_best(double &y, int &idx, float &zf, double y2, int idx2, float zf2) {
   if (idx2 >= 0 && (idx < 0 || y2 > y || (y2 == y && idx2 < idx))) {
     y = y2;
     idx = idx2;
+    zf = zf2;
+  }
+}
+
+__device__ __forceinline__ uint32_t piece_tag(u64 call_id, int j) {
+  return (uint32_t)((((call_id << 4) | (u64)j) * 0x9E3779B97F4A7C15ull) >> 32);
+}
+__device__ __forceinline__ void piece_store(u64 *dst, u64 call_id, const Piece &pc) {
+  uint32_t w[kPieceWords];
+  memcpy(w, &pc, sizeof(Piece));
+#pragma unroll
+  for (int j = 0; j < kPieceWords; ++j) {
+    const u64 v = ((u64)piece_tag(call_id, j) << 32) | w[j];
+    asm volatile("st.relaxed.gpu.global.b64 [%0], %1;" ::"l"(dst + j), "l"(v) : "memory");
+  }
+}
+// False when some word does not carry this call's tag.
+__device__ __forceinline__ bool piece_load(const u64 *src, u64 call_id, Piece &pc) {
+  u64 v[kPieceWords];
+#pragma unroll
+  for (int j = 0; j < kPieceWords; ++j)
+    asm volatile("ld.relaxed.gpu.global.b64 %0, [%1];" : "=l"(v[j]) : "l"(src + j) : "memory");
+  uint32_t w[kPieceWords];
+  bool ok = true;
+#pragma unroll
+  for (int j = 0; j < kPieceWords; ++j) {
+    ok &= (uint32_t)(v[j] >> 32) == piece_tag(call_id, j);
+    w[j] = (uint32_t)v[j];
+  }
+  memcpy(&pc, w, sizeof(Piece));
+  return ok;
+}
+
+// Merges the partial states held by the 32 lanes of a warp; every lane ends with the result.  A lane
+// without weight (Z = 0), without candidate (idx < 0) or with an empty list takes no part.  Written with
+// warp-wide reductions so that the chain of dependent instructions stays short: this runs at the end
+// of every row piece, when nothing else can hide it.  The order of all sums is fixed by lane numbers.
+template <int SAMPLER>
+__device__ __forceinline__ void warp_merge(Piece &pc, Top3 &top, bool with_best) {
+  constexpr unsigned kAll = 0xffffffffu;
+  // softmax sums: move every lane to the largest reference, then add
+  const bool has = pc.Z > 0.f;
+  const int em = __reduce_max_sync(kAll, has ? enc_float(pc.M) : enc_neg_inf());
+  float Mw = 0.f, Zs = 0.f, Ws = 0.f;
+  if (em != enc_neg_inf()) {
+    Mw = dec_float(em);
+    if (has) {
+      const float d = pc.M - Mw, a = ex2f(d);
+      Zs = a * pc.Z;
+      Ws = a * fmaf(d, pc.Z, pc.W);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      Zs += __shfl_xor_sync(kAll, Zs, o);
+      Ws += __shfl_xor_sync(kAll, Ws, o);
+    }
+  }
+  pc.M = Mw; pc.Z = Zs; pc.W = Ws;
+  pc.err = __reduce_or_sync(kAll, pc.err);
+  if (with_best) {
+    // largest y, then lowest index: order-preserving 64-bit code of y, compared half by half
+    const long long bits = __double_as_longlong(pc.y);
+    const long long code = bits >= 0 ? bits : (bits ^ 0x7FFFFFFFFFFFFFFFll);
+    bool cand = pc.idx >= 0;
+    const int hi = cand ? (int)(code >> 32) : INT_MIN;
+    const int hmax = __reduce_max_sync(kAll, hi);
+    if (hmax == INT_MIN) {
+      pc.idx = -1;
+    } else {
+      cand = cand && hi == hmax;
+      const unsigned lo = cand ? (unsigned)code : 0u;
+      const unsigned lmax = __reduce_max_sync(kAll, lo);
+      cand = cand && lo == lmax;
+      const int imin = __reduce_min_sync(kAll, cand ? pc.idx : INT_MAX);
+      const int src = __ffs(__ballot_sync(kAll, cand && pc.idx == imin)) - 1;
+      pc.y = __shfl_sync(kAll, pc.y, src);
+      pc.zf = __shfl_sync(kAll, pc.zf, src);
+      pc.idx = imin;
+    }
+  }
+  if (SAMPLER == 1) {
+    // three rounds of "take the best head": larger score first, equal scores by lower block index
+    Top3 out;
+    top3_reset(out);
+    int pos = 0;
+#pragma unroll
+    for (int r = 0; r < 3; ++r) {
+      const float hy = pos == 0 ? top.y[0] : (pos == 1 ? top.y[1] : top.y[2]);
+      const int hb = pos >= 3 ? -1 : (pos == 0 ? top.b[0] : (pos == 1 ? top.b[1] : top.b[2]));
+      const int e = hb >= 0 ? enc_float(hy) : INT_MIN;
+      const int emax = __reduce_max_sync(kAll, e);
+      if (emax != INT_MIN) {
+        const bool c2 = hb >= 0 && e == emax;
+        const int bmin = __reduce_min_sync(kAll, c2 ? hb : INT_MAX);
+        out.y[r] = dec_float(emax);
+        out.b[r] = bmin;
+        if (c2 && hb == bmin) ++pos;
+      }
+    }
+    top = out;
   }
 }
 
 // ---------------------------------------------------------------------------------------------
 // Work split
 // ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ int64_t quot(const RowsParams &p, int64_t a, int64_t b) {
+  return p.narrow ? (int64_t)((uint32_t)a / (uint32_t)b) : a / b;
+}
 __device__ __forceinline__ int64_t first_tile_of(const RowsParams &p, int64_t b) {
   return b * p.tiles_q + (b < p.tiles_r ? b : p.tiles_r);
 }
 __device__ __forceinline__ int cta_of_tile(const RowsParams &p, int64_t t) {
   const int64_t big = p.tiles_r * (p.tiles_q + 1);
-  return (int)(t < big ? t / (p.tiles_q + 1) : p.tiles_r + (t - big) / p.tiles_q);
+  return (int)(t < big ? quot(p, t, p.tiles_q + 1) : p.tiles_r + quot(p, t - big, p.tiles_q));
 }
 
 struct Walker {
@@ -841,7 +1006,7 @@ struct Walker {
       return true;
     }
     if (t >= t1) return false;
-    const int64_t row = t / p.tiles_per_row, tin = t - row * p.tiles_per_row;
+    const int64_t row = quot(p, t, p.tiles_per_row), tin = t - row * p.tiles_per_row;
     const int64_t n = p.tiles_per_row - tin < t1 - t ? p.tiles_per_row - tin : t1 - t;
     const int64_t lo = tin * kTile, hi = (tin + n) * kTile;
     s.row = row;
@@ -861,17 +1026,38 @@ struct Walker {
   }
 };
 
-__device__ __forceinline__ RowInfo classify(const RowsParams &p, int64_t row) {
-  RowInfo r;
-  r.tau = p.temps ? __ldg(p.temps + row) : p.temp_scalar;
-  const bool sample = p.mode == kModeSample;
-  const bool masked = !sample && p.mask && __ldg(p.mask + row) == 0;
-  r.greedy = sample && r.tau == 0.f;
-  r.invalid = !masked && !r.greedy && !(r.tau > 0.f && r.tau < CUDART_INF_F);
-  r.skip = masked || r.invalid;
-  r.c = r.greedy || r.skip ? 0.f : __fdiv_rn(kLog2e, r.tau);
-  return r;
-}
+// Walks the CTA's row pieces and loads temperature and mask of the piece after the current one, so
+// that nobody waits for them when that piece starts.  The copy-issuing thread passes with_tau = false:
+// it only needs the mask, and must not wait for anything before its first copy.
+struct SegIter {
+  Walker wk;
+  Seg s_next;
+  float tau_next;
+  bool masked_next;
+  bool has;
+  bool with_tau;
+  __device__ SegIter(const RowsParams &p, bool with_tau_) : wk(p), with_tau(with_tau_) { advance(p); }
+  __device__ void advance(const RowsParams &p) {
+    has = wk.next(p, s_next);
+    tau_next = p.temp_scalar;
+    masked_next = false;
+    if (has) {
+      if (with_tau && p.temps) tau_next = __ldg(p.temps + s_next.row);
+      masked_next = p.mode != kModeSample && p.mask && __ldg(p.mask + s_next.row) == 0;
+    }
+  }
+  __device__ bool next(const RowsParams &p, Seg &s, RowInfo &r) {
+    if (!has) return false;
+    s = s_next;
+    r.tau = tau_next;
+    r.masked = masked_next;
+    advance(p);
+    r.greedy = p.mode == kModeSample && r.tau == 0.f;
+    r.invalid = !r.masked && !r.greedy && !(r.tau > 0.f && r.tau < CUDART_INF_F);
+    r.c = r.greedy || r.masked || r.invalid ? 0.f : __fdiv_rn(kLog2e, r.tau);
+    return true;
+  }
+};
 
 template <int DT>
 __device__ __forceinline__ const char *row_ptr(const RowsParams &p, int64_t row) {
@@ -879,11 +1065,11 @@ __device__ __forceinline__ const char *row_ptr(const RowsParams &p, int64_t row)
 }
 
 // ---------------------------------------------------------------------------------------------
-// Row epilogue (one thread, fp64)
+// Row epilogue (one thread, fp64).  zt: logit of the token whose log-probability is wanted.
 // ---------------------------------------------------------------------------------------------
-template <int DT>
-__device__ __forceinline__ void finish_row(const RowsParams &p, int64_t row, const RowInfo &ri, double M, double Z,
-                                           double W, double y, int idx, int err) {
+__device__ __forceinline__ void finish_row(const RowsParams &p, int64_t row, const RowInfo &ri, float Mf, float Zf,
+                                           float Wf, int idx, int err, bool have_zt, float zt) {
+  const double M = Mf, Z = Zf, W = Wf;
   const bool sample = p.mode == kModeSample;
   int tok = -1;
   float logp = CUDART_NAN_F, ent = CUDART_NAN_F;
@@ -892,12 +1078,8 @@ __device__ __forceinline__ void finish_row(const RowsParams &p, int64_t row, con
   } else if (err == 0 && Z > 0.0) {
     const double lnZ = log(Z);
     ent = (float)(lnZ - kLn2 * (W / Z));
-    const int t = sample ? idx : __ldg(p.targets + row);
-    if (sample) tok = t;
-    if (t >= 0 && t < p.V) {
-      const double zt = (double)load_elem<DT>(row_ptr<DT>(p, row), t);
-      logp = (float)((zt * (double)ri.c - M) * kLn2 - lnZ);
-    }
+    if (sample) tok = idx;
+    if (have_zt) logp = (float)(((double)zt * (double)ri.c - M) * kLn2 - lnZ);
   }
   if (sample) p.out_tok[row] = tok;
   if (p.out_logp) p.out_logp[row] = logp;
@@ -954,8 +1136,9 @@ __device__ __noinline__ double exact_block_score(const EvalCtx &x, int b, int la
 }
 
 // Token inside block b: first entry whose inclusive prefix sum of exp(s_i - m_b) exceeds v * total.
+// Exact form (fp64, the definition's expression order).
 template <int DT>
-__device__ __noinline__ int draw_in_block(const EvalCtx &x, int b, int lane) {
+__device__ __noinline__ int draw_in_block_exact(const EvalCtx &x, int b, int lane) {
   BlockView v;
   load_block<DT>(x.row, b, x.V, (double)x.tau, lane, v);
   double pre[8];
@@ -996,10 +1179,74 @@ __device__ __noinline__ int draw_in_block(const EvalCtx &x, int b, int lane) {
   return tok;
 }
 
+// The same draw in fp32.  When the threshold comes closer than 1e-4 of the block sum to a prefix
+// boundary (fp32 prefix sums are good to about 1e-5) the exact form decides.  z_tok: logit of the token.
+template <int DT>
+__device__ __noinline__ int draw_in_block(const EvalCtx &x, int b, int lane, float &z_tok) {
+  float z[8];
+  float m = -CUDART_INF_F;
+#pragma unroll
+  for (int k = 0; k < 8; ++k) {
+    const int i = b * 256 + lane * 8 + k;
+    z[k] = i < x.V ? load_elem<DT>(x.row, i) : -CUDART_INF_F;
+    m = fmaxf(m, z[k]);
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+  int tok = -1;
+  bool exact = !(m > -CUDART_INF_F && m < CUDART_INF_F);
+  if (!exact) {
+    const float c = __fdiv_rn(kLog2e, x.tau);
+    float pre[8];
+    float run = 0.f;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+      run += z[k] > -CUDART_INF_F ? ex2f((z[k] - m) * c) : 0.f;
+      pre[k] = run;
+    }
+    float incl = run;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const float up = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += up;
+    }
+    const float total = __shfl_sync(0xffffffffu, incl, 31);
+    const float before = incl - run;
+    const uint4 w3 = philox(x.rk, 0u, x.grow, x.ctr_lo, x.ctr_hi8 | 3u);
+    const float t = (float)((((double)w3.x + 0.5) * 0x1p-32) * (double)total);
+    int hit = -1;
+    float gap = CUDART_INF_F;
+#pragma unroll
+    for (int k = 7; k >= 0; --k) {
+      const float pk = before + pre[k];
+      if (pk > t) hit = k;
+      gap = fminf(gap, fabsf(pk - t));
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) gap = fminf(gap, __shfl_xor_sync(0xffffffffu, gap, o));
+    const uint32_t found = __ballot_sync(0xffffffffu, hit >= 0);
+    exact = !(gap > 1e-4f * total) || found == 0u || !(total > 0.f) || !(total < CUDART_INF_F);
+    if (!exact) {
+      const int src = __ffs(found) - 1;
+      const int k = __shfl_sync(0xffffffffu, hit, src);
+      tok = b * 256 + src * 8 + k;
+      float zk = z[0];
+#pragma unroll
+      for (int j = 1; j < 8; ++j) zk = k == j ? z[j] : zk;
+      z_tok = __shfl_sync(0xffffffffu, zk, src);
+    }
+  }
+  if (exact) {
+    tok = draw_in_block_exact<DT>(x, b, lane);
+    z_tok = tok >= 0 ? load_elem<DT>(x.row, tok) : 0.f;
+  }
+  return tok;
+}
+
 // Picks the winning block from the three fp32 leaders (exact scores where they are too close) and
 // draws the token.  Returns -1 when the row has no block with mass.
 template <int DT>
-__device__ __noinline__ int sample_in_blocks(const EvalCtx &x, const Top3 &top, int lane) {
+__device__ __noinline__ int sample_in_blocks(const EvalCtx &x, const Top3 &top, int lane, float &z_tok) {
   if (top.b[0] < 0) return -1;
   int bstar = top.b[0];
   const float margin = 1e-4f + 2e-5f * fabsf(top.y[0]);
@@ -1019,7 +1266,7 @@ __device__ __noinline__ int sample_in_blocks(const EvalCtx &x, const Top3 &top, 
     }
     if (bbest >= 0) bstar = bbest;
   }
-  return draw_in_block<DT>(x, bstar, lane);
+  return draw_in_block<DT>(x, bstar, lane, z_tok);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -1027,12 +1274,16 @@ __device__ __noinline__ int sample_in_blocks(const EvalCtx &x, const Top3 &top, 
 // ---------------------------------------------------------------------------------------------
 template <int DT, int SAMPLER, bool RING>
 __global__ void __launch_bounds__(kThreads, 2) rows_kernel(const __grid_constant__ RowsParams p) {
-  extern __shared__ __align__(128) unsigned char ring[];
+  extern __shared__ __align__(128) unsigned char dyn[];  // ring, then the candidate queues of sampler 0
   __shared__ Smem sm;
-  constexpr int kEsize = DT == 0 ? 4 : 2;
-  constexpr int kChunkE = kStageBytes / kEsize;                    // entries per stage: 8,192 bf16 / 4,096 fp32
-  constexpr int kGPT = kChunkE / (kStreamThreads * kGroup);        // 16-entry groups per consumer thread and stage
+  using F = Fmt<DT>;
+  constexpr int kEsize = F::kEsize;
+  constexpr int kChunkE = F::kChunkE;
+  constexpr int kLaneE = F::kLaneE;
+  constexpr int kG = F::kG;
+  constexpr int kVG = F::kVG;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  unsigned char *const ring = dyn;
 
   if (tid == 0) {
     for (int s = 0; s < kStages; ++s) { mbar_init(&sm.full[s], 1); mbar_init(&sm.empty[s], kStreamWarps); }
@@ -1047,174 +1298,258 @@ __global__ void __launch_bounds__(kThreads, 2) rows_kernel(const __grid_constant
 
   if (warp < kStreamWarps) {
     // ------------------------------------------------------------------ consumers
-    Walker wk(p);
+    SegIter it(p, true);
     Seg s;
+    RowInfo ri;
     uint32_t stage = 0, phase = 0;  // ring position
     uint32_t n = 0;                 // segments handed to the finishing warp so far
-    while (wk.next(p, s)) {
-      const RowInfo ri = classify(p, s.row);
-      if (ri.skip) continue;
+    const uint32_t *const rk = p.round_key;
+    unsigned char *const queue = dyn + (RING ? kStages * kStageBytes : 0) + warp * F::kQueueBytes;
+    // vector order of this lane inside its 64 bytes (the lanes of a quarter warp hit distinct banks)
+    const int rot = (lane >> 1) & 3;
+    while (it.next(p, s, ri)) {
+      if (ri.masked) continue;
+      if (ri.invalid) {
+        // nothing to compute, but the row's chunks are on their way: let them pass
+        if (RING) {
+          const int nc = s.e_hi > s.e_lo ? (s.e_hi - s.e_lo + kChunkE - 1) / kChunkE : 0;
+          for (int c = 0; c < nc; ++c) {
+            mbar_wait(&sm.full[stage], phase, sm);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sm.empty[stage]);
+            if (++stage == kStages) { stage = 0; phase ^= 1u; }
+          }
+        }
+        continue;
+      }
       const char *row = row_ptr<DT>(p, s.row);
-      EvalCtx ex;
-      ex.rk = p.round_key; ex.row = row; ex.tau = ri.tau; ex.grow = p.row_base + (uint32_t)s.row;
-      ex.ctr_lo = p.ctr_lo; ex.ctr_hi8 = p.ctr_hi8; ex.seg = n + 1; ex.V = (int)p.V;
+      const uint32_t grow = p.row_base + (uint32_t)s.row;
+      const uint32_t seg = n + 1;
+#define E3_MAKE_CTX(ex)                                                                                  \
+  EvalCtx ex;                                                                                            \
+  ex.rk = rk; ex.row = row; ex.tau = ri.tau; ex.grow = grow; ex.ctr_lo = p.ctr_lo; ex.ctr_hi8 = p.ctr_hi8; \
+  ex.seg = seg; ex.V = (int)p.V
 
       Acc acc;
+      acc_reset(acc);
       Best best;
-      int err, qn = 0;
-      acc.R = -CUDART_INF_F; acc.nRc = kNoRef; acc.Z0 = acc.Z1 = acc.W0 = acc.W1 = 0.f;
-      best.y = -CUDART_INF; best.idx = -1;
+      best.y = -CUDART_INF; best.idx = -1; best.zf = 0.f;
       set_gate(best, enc_neg_inf(), ri.tau);
-      err = 0;
+      float ethr = 0.f;
+      int err = 0, qn = 0;
       BlockState bs;
       block_state_reset(bs);
 
       const int nchunks = s.e_hi > s.e_lo ? (s.e_hi - s.e_lo + kChunkE - 1) / kChunkE : 0;
-      const int fast_end = s.e_hi < full_end ? s.e_hi : full_end;  // chunks ending at or before this are full
-      if (RING && SAMPLER == 0 && !ri.greedy && nchunks > 0) {
-        // seed the gate from the first stage of the segment (the stage is consumed by the loop below)
-        mbar_wait(&sm.full[stage], phase, sm);
-        const int e0 = s.e_lo + tid * kGroup;
-        seed_from_stage<DT>(ex, ring + (size_t)stage * kStageBytes, tid, e0, e0 + kGroup <= fast_end, best, sm);
-      }
+      const int fast_end = s.e_hi < full_end ? s.e_hi : full_end;  // full groups of the piece end here
+      const bool stream = RING && !ri.greedy;
 #pragma unroll 1
       for (int c = 0; c < nchunks; ++c) {
         const int cs = s.e_lo + c * kChunkE;
+        const int e_lane = cs + tid * kLaneE;
         const unsigned char *stage_ptr = nullptr;
         if (RING) {
           mbar_wait(&sm.full[stage], phase, sm);
           stage_ptr = ring + (size_t)stage * kStageBytes;
         }
-        if (SAMPLER == 0 && !ri.greedy) {
-          const int enc = read_best(sm, ex.seg);
-          if (enc > best.enc) set_gate(best, enc, ri.tau);
-        }
-        if (SAMPLER == 1 && !ri.greedy) {
-          if (RING && cs + kChunkE <= fast_end) {
-#pragma unroll
-            for (int j = 0; j < kGPT; ++j) {
-              const int slot = j * kStreamThreads + tid;
-              hot_group_blocks<DT>(ex, stage_ptr, slot, cs + slot * kGroup, ri.c, acc, bs, err, lane);
+        if (stream) {
+          const unsigned char *lane_data = stage_ptr + tid * kLaneBytes;
+          const int lim = fast_end < cs + kChunkE ? fast_end : cs + kChunkE;
+          if (c == 0) {
+            SeedIO sd;
+            sd.best = best;
+            E3_MAKE_CTX(ex);
+            seed_piece<DT, SAMPLER>(sd, ex, lane_data, e_lane, lim, sm);
+            best = sd.best;
+            if (sd.R0 > -CUDART_INF_F) {
+              const float nRc = -sd.R0 * ri.c;
+              if (fabsf(nRc) < CUDART_INF_F) { acc.R = sd.R0; acc.nRc = nRc; }
             }
-          } else {
-            LaneStateBlocks st;
-            st.acc = acc; st.bs = bs; st.err = err;
-#pragma unroll 1
-            for (int j = 0; j < kGPT; ++j)
-              slow_group_blocks<DT>(ex, stage_ptr, j * kStreamThreads + tid, cs, s.e_hi, ri.c, st);
-            acc = st.acc; bs = st.bs; err = st.err;
-          }
-        } else if (RING && !ri.greedy) {
-          const bool all_full = cs + kChunkE <= fast_end;
-#pragma unroll
-          for (int j = 0; j < kGPT; ++j) {
-            const int slot = j * kStreamThreads + tid;
-            const int e0 = cs + slot * kGroup;
-            hot_group<DT, SAMPLER>(ex, stage_ptr, slot, e0, ri.c, all_full || e0 + kGroup <= fast_end, acc, best, err,
-                                   qn, sm, warp, lane);
-          }
-          // the row's last, partial group (V not a multiple of 16) goes through the out-of-line path
-          if (!all_full && fast_end < s.e_hi && fast_end >= cs && fast_end < cs + kChunkE) {
-            const int slot = (fast_end - cs) / kGroup;
-            if (((slot % kStreamThreads) >> 5) == warp) {
-              LaneState st;
-              st.acc = acc; st.best = best; st.err = err; st.qn = qn;
-              // only the owning lane has the group; the others pass an empty range
-              slow_group<DT, SAMPLER>(ex, nullptr, slot, cs, (slot % kStreamThreads) == tid ? s.e_hi : 0, ri.c, false,
-                                      false, st, sm);
-              acc = st.acc; best = st.best; err = st.err; qn = st.qn;
+            if (SAMPLER == 0) ethr = gate_threshold(best.enc, acc.nRc);
+          } else if (SAMPLER == 0 && (c & 3) == 0) {
+            const int enc = read_best(sm, seg);
+            if (enc > best.enc) {
+              set_gate(best, enc, ri.tau);
+              ethr = gate_threshold(best.enc, acc.nRc);
             }
           }
+          // the row's last, partial group (V not a multiple of 16) sits behind the full groups of this chunk
+          float zextra = 0.f;
+          const bool tail_here = fast_end < s.e_hi && fast_end >= cs && fast_end < cs + kChunkE;
+          if (tail_here) {
+            const int owner = (fast_end - cs) / kLaneE;  // thread whose 64 bytes would hold it
+            if ((owner >> 5) == warp) {
+              SlowIO io;
+              io.acc = acc; io.best = best; io.err = err; io.zsum = 0.f;
+              E3_MAKE_CTX(ex);
+              slow_groups<DT, SAMPLER, SAMPLER == 1>(io, ex, owner == tid ? fast_end : s.e_hi, s.e_hi, ri.c, sm);
+              acc = io.acc; best = io.best; err = io.err;
+              zextra = io.zsum;
+              if (SAMPLER == 0) ethr = gate_threshold(best.enc, acc.nRc);
+            }
+          }
+          // ---- the streaming form
+          uint4 raw[4];
+          {
+            const uint4 *pv = reinterpret_cast<const uint4 *>(lane_data);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) raw[i] = pv[i ^ rot];
+          }
+          // raw[kVG*gi ...] is group gi ^ ga of the thread (vocabulary order)
+          const int ga = kG == 2 ? (rot >> 1) : 0;
+          const Acc saved = acc;
+          const u64 c2 = pack2f(ri.c, ri.c), nRc2 = pack2f(acc.nRc, acc.nRc);
+          float Zg[kG];
+          bool have[kG];
+          bool bad = false;
+#pragma unroll
+          for (int gi = 0; gi < kG; ++gi) {
+            const int g0 = e_lane + ((gi ^ ga) << 4);
+            have[gi] = g0 + kGroup <= lim;
+            Zg[gi] = 0.f;
+            if (have[gi]) {
+              u64 Zg2;
+              Zg[gi] = hot_group<DT>(&raw[kVG * gi], c2, nRc2, acc.Wa2, acc.Wb2, Zg2);
+              acc.Z2 = add2(acc.Z2, Zg2);
+              bad |= !(Zg[gi] <= kGroupSumMax);
+            }
+          }
+          if (SAMPLER == 1) bad = __any_sync(0xffffffffu, bad);
+          if (bad) {
+            StepIO io;
+            io.acc = saved; io.err = err; io.Zextra = zextra;
+            io.Zg[0] = 0.f; io.Zg[kG - 1] = 0.f;
+            int hv = 0;
+#pragma unroll
+            for (int gi = 0; gi < kG; ++gi) hv |= (have[gi] ? 1 : 0) << (gi ^ ga);
+            redo_step<DT, SAMPLER == 1>(io, lane_data, hv, ri.c);
+            acc = io.acc; err = io.err; zextra = io.Zextra;
+#pragma unroll
+            for (int gi = 0; gi < kG; ++gi) Zg[gi] = io.Zg[gi ^ ga];
+            if (SAMPLER == 0) ethr = gate_threshold(best.enc, acc.nRc);
+          }
+          if (SAMPLER == 0) {
+#pragma unroll
+            for (int gi = 0; gi < kG; ++gi) {
+              const int g0 = e_lane + ((gi ^ ga) << 4);
+              const uint4 cb = philox(rk, (uint32_t)g0 >> 4, grow, p.ctr_lo, p.ctr_hi8 | 0u);
+              const bool over = Zg[gi] > ethr;
+              const bool flag = have[gi] && (any_ff4(cb) != 0u || over);
+              const uint32_t ballot = __ballot_sync(0xffffffffu, flag);
+              if (ballot != 0u) {
+                if (flag) {
+                  const int pos = qn + __popc(ballot & ((1u << lane) - 1u));
+                  reinterpret_cast<int *>(queue)[pos] = g0 | (over ? 1 : 0);
+                  uint4 *ent = reinterpret_cast<uint4 *>(queue + kQueueHdrBytes + pos * F::kEntryBytes);
+                  ent[0] = cb;
+#pragma unroll
+                  for (int i = 0; i < kVG; ++i) ent[1 + ((i ^ rot) & (kVG - 1))] = raw[kVG * gi + i];
+                }
+                qn += __popc(ballot);
+                if (qn >= kDrainAt) {
+                  Best tb = best;
+                  E3_MAKE_CTX(ex);
+                  drain_queue<DT>(ex, tb, sm, queue, qn);
+                  best = tb;
+                  qn = 0;
+                  const int enc = read_best(sm, seg);
+                  if (enc > best.enc) set_gate(best, enc, ri.tau);
+                  ethr = gate_threshold(best.enc, acc.nRc);
+                }
+              }
+            }
+          }
+          if (SAMPLER == 1) {
+            float zl = zextra;
+#pragma unroll
+            for (int gi = 0; gi < kG; ++gi) zl += Zg[gi];
+            block_step<DT>(zl, e_lane >> 8, acc.nRc, rk, grow, p.ctr_lo, p.ctr_hi8, bs, lane);
+          }
+        } else if (ri.greedy) {
+          SlowIO io;
+          io.acc = acc; io.best = best; io.err = err; io.zsum = 0.f;
+          greedy_groups<DT>(io, row, RING ? stage_ptr + tid * kLaneBytes : nullptr, e_lane,
+                            fast_end < cs + kChunkE ? fast_end : cs + kChunkE, s.e_hi);
+          best = io.best; err = io.err;
         } else {
-          // the out-of-line path works on a copy, so that the streaming loop keeps its state in registers
-          LaneState st;
-          st.acc = acc; st.best = best; st.err = err; st.qn = qn;
-#pragma unroll 1
-          for (int j = 0; j < kGPT; ++j)
-            slow_group<DT, SAMPLER>(ex, stage_ptr, j * kStreamThreads + tid, cs, s.e_hi, ri.c, ri.greedy,
-                                    !RING && SAMPLER == 0 && !ri.greedy && c == 0 && j == 0, st, sm);
-          acc = st.acc; best = st.best; err = st.err; qn = st.qn;
+          // rows that cannot use the ring: everything through the guarded form
+          SlowIO io;
+          io.acc = acc; io.best = best; io.err = err; io.zsum = 0.f;
+          E3_MAKE_CTX(ex);
+          slow_groups<DT, SAMPLER, SAMPLER == 1>(io, ex, e_lane < s.e_hi ? e_lane : s.e_hi, s.e_hi, ri.c, sm);
+          acc = io.acc; best = io.best; err = io.err;
+          if (SAMPLER == 1) block_step<DT>(io.zsum, e_lane >> 8, acc.nRc, rk, grow, p.ctr_lo, p.ctr_hi8, bs, lane);
         }
         if (RING) {
           __syncwarp();
           if (lane == 0) mbar_arrive(&sm.empty[stage]);
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
-        // All warps of the CTA drain at the same chunks: a drain stalls its warp for microseconds and the
-        // ring moves at the pace of the slowest warp, so staggered drains would add up.
-        if (SAMPLER == 0 && qn > 0 && ((c & (kDrainEvery - 1)) == kDrainEvery - 1 || qn > kQueueCap - 32 * kGPT))
-          drain_queue<DT>(ex, best, sm, warp, lane, qn, RING);
       }
-      if (SAMPLER == 0 && qn > 0) drain_queue<DT>(ex, best, sm, warp, lane, qn, RING);
-      if (SAMPLER == 1 && !ri.greedy) block_flush(ex, bs);
+      if (SAMPLER == 0 && qn > 0) {
+        Best tb = best;
+        E3_MAKE_CTX(ex);
+        drain_queue<DT>(ex, tb, sm, queue, qn);
+        best = tb;
+        qn = 0;
+      }
+      if (SAMPLER == 1 && !ri.greedy) {
+        BlockState t = bs;
+        block_flush(rk, grow, p.ctr_lo, p.ctr_hi8, t);
+        bs = t;
+      }
 
+      AccS fin = to_scalar(acc);
       if (!ri.greedy) {
-        // -inf or NaN logits poison the fast sums: redo this warp's groups with the careful form
-        const float zs = acc.Z0 + acc.Z1, ws = acc.W0 + acc.W1;
-        const bool bad = !(fabsf(zs) < CUDART_INF_F) || !(fabsf(ws) < CUDART_INF_F);
-        if (__any_sync(0xffffffffu, bad)) {
-          acc.R = -CUDART_INF_F; acc.nRc = kNoRef; acc.Z0 = acc.Z1 = acc.W0 = acc.W1 = 0.f;
+        // NaN or infinite sums (a NaN or +inf logit, or numbers outside the fp32 range): settle this
+        // thread's entries of the piece with the careful form, which also says what was wrong
+        const bool odd = !(fabsf(fin.Z) < CUDART_INF_F) || !(fabsf(fin.W) < CUDART_INF_F);
+        if (__any_sync(0xffffffffu, odd)) {
+          fin.R = -CUDART_INF_F; fin.nRc = kNoRef; fin.Z = fin.W = 0.f;
 #pragma unroll 1
-          for (int c = 0; c < nchunks * kGPT; ++c) {
-            const int e0 = s.e_lo + (c * kStreamThreads + tid) * kGroup;
+          for (int g = 0; g < nchunks * kG; ++g) {
+            const int e0 = s.e_lo + (g / kG) * kChunkE + tid * kLaneE + (g % kG) * kGroup;
             if (e0 < s.e_hi) {
               float z[16];
-              const float gmax = load_group_guarded<DT>(row, e0, e0 + kGroup <= (int)p.V ? 16 : (int)p.V - e0, z);
-              accumulate<true>(acc, z, ri.c, gmax, err);
+              load_group_guarded<DT>(row, e0, e0 + kGroup <= (int)p.V ? 16 : (int)p.V - e0, z);
+              careful_accumulate(fin, z, ri.c, -CUDART_INF_F, err);
             }
           }
         }
       }
 
       // warp-level merge, hand-over to the finishing warp
-      float M = -acc.nRc, Z = acc.Z0 + acc.Z1, W = acc.W0 + acc.W1;
-      if (acc.R == -CUDART_INF_F) { M = 0.f; Z = 0.f; W = 0.f; }
-      double y = best.y;
-      int idx = best.idx;
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) {
-        const float M2 = __shfl_xor_sync(0xffffffffu, M, o), Z2 = __shfl_xor_sync(0xffffffffu, Z, o),
-                    W2 = __shfl_xor_sync(0xffffffffu, W, o);
-        const double y2 = __shfl_xor_sync(0xffffffffu, y, o);
-        const int idx2 = __shfl_xor_sync(0xffffffffu, idx, o);
-        err |= __shfl_xor_sync(0xffffffffu, err, o);
-        merge_stats_f(M, Z, W, M2, Z2, W2);
-        merge_best(y, idx, y2, idx2);
-        if (SAMPLER == 1) {
-          Top3 o2;
-#pragma unroll
-          for (int i = 0; i < 3; ++i) {
-            o2.y[i] = __shfl_xor_sync(0xffffffffu, bs.top.y[i], o);
-            o2.b[i] = __shfl_xor_sync(0xffffffffu, bs.top.b[i], o);
-          }
-          top3_merge(bs.top, o2);
-        }
-      }
+      Piece pw;
+      pw.M = -fin.nRc; pw.Z = fin.Z; pw.W = fin.W;
+      if (fin.R == -CUDART_INF_F) { pw.M = 0.f; pw.Z = 0.f; pw.W = 0.f; }
+      pw.y = best.y; pw.idx = best.idx; pw.zf = best.zf; pw.err = err;
+      warp_merge<SAMPLER>(pw, bs.top, p.mode == kModeSample);
       const uint32_t slot = n % kSlots, use = n / kSlots;
       if (use > 0) mbar_wait(&sm.wfree[slot], (use - 1) & 1u, sm);
       if (lane == 0) {
         WarpPartial &w = sm.wpart[slot][warp];
-        w.M = M; w.Z = Z; w.W = W; w.y = y; w.idx = idx; w.err = err;
+        w.M = pw.M; w.Z = pw.Z; w.W = pw.W; w.y = pw.y; w.idx = pw.idx; w.err = pw.err; w.zf = pw.zf;
 #pragma unroll
         for (int i = 0; i < 3; ++i) { w.ty[i] = bs.top.y[i]; w.tb[i] = bs.top.b[i]; }
         mbar_arrive(&sm.wfull[slot]);
       }
       ++n;
     }
+#undef E3_MAKE_CTX
   } else if (warp == kStreamWarps) {
     // ------------------------------------------------------------------ producer (one thread)
     if (RING && lane == 0) {
-      Walker wk(p);
+      SegIter it(p, false);
       Seg s;
+      RowInfo ri;
       uint32_t cc = 0, stage = 0, phase = 1;  // phase: parity of the previous use of the stage
-      while (wk.next(p, s)) {
-        const RowInfo ri = classify(p, s.row);
-        if (ri.skip) continue;
+      while (it.next(p, s, ri)) {
+        if (ri.masked) continue;
         const char *row = row_ptr<DT>(p, s.row);
         const int nchunks = s.e_hi > s.e_lo ? (s.e_hi - s.e_lo + kChunkE - 1) / kChunkE : 0;
         const int lim = s.e_hi < full_end ? s.e_hi : full_end;
         for (int c = 0; c < nchunks; ++c) {
-          if (cc >= (uint32_t)kStages) mbar_wait(&sm.empty[stage], phase, sm, 200u);
+          if (cc >= (uint32_t)kStages) mbar_wait(&sm.empty[stage], phase, sm, 32u);
           const int cs = s.e_lo + c * kChunkE;
           const int ce = cs + kChunkE < lim ? cs + kChunkE : lim;
           const uint32_t bytes = ce > cs ? (uint32_t)(ce - cs) * kEsize : 0u;
@@ -1232,31 +1567,40 @@ __global__ void __launch_bounds__(kThreads, 2) rows_kernel(const __grid_constant
       // Before leaving, see every copy still in flight land (bounded).
       const uint32_t back = cc < (uint32_t)kStages ? cc : (uint32_t)kStages;
       for (uint32_t q = cc - back; q < cc; ++q) {
-        const uint32_t stage = q % kStages, round = q / kStages;
-        for (uint32_t it = 0; it < kSpinLimit && !mbar_try_wait(&sm.full[stage], round & 1u); ++it) __nanosleep(64);
+        const uint32_t st = q % kStages, round = q / kStages;
+        for (uint32_t i = 0; i < kSpinLimit && !mbar_try_wait(&sm.full[st], round & 1u); ++i) __nanosleep(64);
       }
     }
   } else {
     // ------------------------------------------------------------------ finishing warp
-    Walker wk(p);
+    SegIter it(p, true);
     Seg s;
+    RowInfo ri;
     uint32_t n = 0;
-    Piece *pieces = reinterpret_cast<Piece *>(p.ws_pieces);
-    while (wk.next(p, s)) {
-      const RowInfo ri = classify(p, s.row);
-      if (ri.skip) {
+    u64 *const pieces = reinterpret_cast<u64 *>(p.ws_pieces);
+    constexpr int kPieceStride = (int)(kPieceBytes / 8);
+    const bool sample = p.mode == kModeSample;
+    while (it.next(p, s, ri)) {
+      if (ri.masked || ri.invalid) {
         if (s.starts && lane == 0) write_skipped(p, s.row, ri);
         continue;
       }
+      // the target's logit is fetched while the consumers work on the piece
+      int target = -1;
+      float zt = 0.f;
+      if (!sample && lane == 0) {
+        target = __ldg(p.targets + s.row);
+        if (target >= 0 && target < p.V) zt = load_elem<DT>(row_ptr<DT>(p, s.row), target);
+      }
       const uint32_t slot = n % kSlots, use = n / kSlots;
       mbar_wait_warp(&sm.wfull[slot], use & 1u, sm, lane);
-      double Md = 0.0, Zd = 0.0, Wd = 0.0, yd = -CUDART_INF;
-      int id = -1, ed = 0;
+      Piece pc;
+      pc.y = -CUDART_INF; pc.M = 0.f; pc.Z = 0.f; pc.W = 0.f; pc.idx = -1; pc.zf = 0.f; pc.err = 0;
       Top3 top;
       top3_reset(top);
       if (lane < kStreamWarps) {
         const WarpPartial &w = sm.wpart[slot][lane];
-        Md = w.M; Zd = w.Z; Wd = w.W; yd = w.y; id = w.idx; ed = w.err;
+        pc.M = w.M; pc.Z = w.Z; pc.W = w.W; pc.y = w.y; pc.idx = w.idx; pc.err = w.err; pc.zf = w.zf;
         if (SAMPLER == 1) {
 #pragma unroll
           for (int i = 0; i < 3; ++i) { top.y[i] = w.ty[i]; top.b[i] = w.tb[i]; }
@@ -1265,84 +1609,62 @@ __global__ void __launch_bounds__(kThreads, 2) rows_kernel(const __grid_constant
       __syncwarp();
       if (lane == 0) mbar_arrive(&sm.wfree[slot]);
       ++n;
+      // The order of every merge below is fixed by lane and piece numbers alone, so the result does not
+      // depend on which CTA ends up finishing the row.
+      warp_merge<SAMPLER>(pc, top, sample);
+      if (*reinterpret_cast<volatile int *>(&sm.timeout)) pc.err |= kErrTimeout;
+      bool fin = s.whole;
+      if (!s.whole) {
+        // A piece of a cut row.  Store it, then (after a sequentially consistent fence) look for the
+        // row's other pieces: of all CTAs that hold a piece, the one whose fence comes last is sure to
+        // find them all and finishes the row.  Two CTAs may both find all pieces; they then write the
+        // same values.  Nobody waits for anybody.
+        if (lane == 0) {
 #pragma unroll
-      for (int o = kStreamWarps / 2; o > 0; o >>= 1) {
-        const double M2 = __shfl_xor_sync(0xffffffffu, Md, o), Z2 = __shfl_xor_sync(0xffffffffu, Zd, o),
-                     W2 = __shfl_xor_sync(0xffffffffu, Wd, o), y2 = __shfl_xor_sync(0xffffffffu, yd, o);
-        const int i2 = __shfl_xor_sync(0xffffffffu, id, o);
-        ed |= __shfl_xor_sync(0xffffffffu, ed, o);
-        merge_stats_d(Md, Zd, Wd, M2, Z2, W2);
-        merge_best(yd, id, y2, i2);
-        if (SAMPLER == 1) {
-          Top3 o2;
-#pragma unroll
-          for (int i = 0; i < 3; ++i) {
-            o2.y[i] = __shfl_xor_sync(0xffffffffu, top.y[i], o);
-            o2.b[i] = __shfl_xor_sync(0xffffffffu, top.b[i], o);
-          }
-          top3_merge(top, o2);
+          for (int i = 0; i < 3; ++i) { pc.ty[i] = top.y[i]; pc.tb[i] = top.b[i]; }
+          piece_store(pieces + ((size_t)blockIdx.x * 2 + (s.first ? 0 : 1)) * kPieceStride, p.call_id, pc);
+          asm volatile("fence.sc.gpu;" ::: "memory");
         }
-      }
-      // lane 0 runs the piece protocol and decides whether this CTA finishes the row
-      int fin = 0;
-      if (lane == 0) {
-        if (*reinterpret_cast<volatile int *>(&sm.timeout)) ed |= kErrTimeout;
-        if (s.whole) {
-          fin = 1;
-        } else {
-          // A piece of a cut row: store it, announce it; whoever completes the row finishes it.
-          Piece *mine = pieces + (size_t)blockIdx.x * 2 + (s.first ? 0 : 1);
-          mine->M = Md; mine->Z = Zd; mine->W = Wd; mine->y = yd; mine->idx = id; mine->err = ed;
-#pragma unroll
-          for (int i = 0; i < 3; ++i) { mine->ty[i] = top.y[i]; mine->tb[i] = top.b[i]; }
-          __threadfence();
-          const unsigned long long tag = p.call_id << 16;
-          unsigned long long *word = p.ws_arrivals + s.k0;
-          unsigned long long cur = *reinterpret_cast<volatile unsigned long long *>(word), want = 0;
-          bool done = false;
-          for (int it = 0; it < 65536 && !done; ++it) {  // lock-free: some contender always gets through
-            want = (cur >> 16) == p.call_id ? cur + 1 : (tag | 1ull);
-            const unsigned long long prev = atomicCAS(word, cur, want);
-            done = prev == cur;
-            cur = prev;
+        __syncwarp();
+        pc.y = -CUDART_INF; pc.M = 0.f; pc.Z = 0.f; pc.W = 0.f; pc.idx = -1; pc.zf = 0.f; pc.err = 0;
+        top3_reset(top);
+        bool ok = true;
+        for (int k = s.k0 + lane; k <= s.k1; k += 32) {
+          // CTA k keeps this row's piece in slot 0 when the row is the first thing it works on
+          const bool is_first_seg = quot(p, first_tile_of(p, k), p.tiles_per_row) == s.row;
+          Piece q;
+          if (!piece_load(pieces + ((size_t)k * 2 + (is_first_seg ? 0 : 1)) * kPieceStride, p.call_id, q)) {
+            ok = false;
+            break;
           }
-          if (done && (int)(want & 0xFFFFull) == s.k1 - s.k0 + 1) {  // the last piece of the row
-            __threadfence();
-            Md = 0.0; Zd = 0.0; Wd = 0.0; yd = -CUDART_INF; id = -1; ed = 0;
-            top3_reset(top);
-            for (int k = s.k0; k <= s.k1; ++k) {
-              // CTA k keeps this row's piece in slot 0 when the row is the first thing it works on
-              const bool is_first_seg = first_tile_of(p, k) / p.tiles_per_row == s.row;
-              const volatile Piece *q = pieces + (size_t)k * 2 + (is_first_seg ? 0 : 1);
-              const double M2 = q->M, Z2 = q->Z, W2 = q->W, y2 = q->y;
-              const int i2 = q->idx;
-              ed |= q->err;
-              merge_stats_d(Md, Zd, Wd, M2, Z2, W2);
-              merge_best(yd, id, y2, i2);
-              if (SAMPLER == 1) {
+          pc.err |= q.err;
+          merge_stats_f(pc.M, pc.Z, pc.W, q.M, q.Z, q.W);
+          merge_best(pc.y, pc.idx, pc.zf, q.y, q.idx, q.zf);
+          if (SAMPLER == 1) {
 #pragma unroll
-                for (int i = 0; i < 3; ++i) top3_insert(top, q->ty[i], q->tb[i]);
-              }
-            }
-            fin = 1;
+            for (int i = 0; i < 3; ++i) top3_insert(top, q.ty[i], q.tb[i]);
           }
         }
+        fin = __all_sync(0xffffffffu, ok);
+        if (fin) warp_merge<SAMPLER>(pc, top, sample);
       }
-      fin = __shfl_sync(0xffffffffu, fin, 0);
       if (!fin) continue;
-      if (SAMPLER == 1 && !ri.greedy) {
-        // the whole warp settles the block and draws inside it
-#pragma unroll
-        for (int i = 0; i < 3; ++i) {
-          top.y[i] = __shfl_sync(0xffffffffu, top.y[i], 0);
-          top.b[i] = __shfl_sync(0xffffffffu, top.b[i], 0);
+      int id = pc.idx;
+      bool have_zt = !sample && target >= 0 && target < p.V;
+      if (sample && !ri.greedy) {
+        if (SAMPLER == 1) {
+          // the whole warp settles the block and draws inside it
+          EvalCtx ex;
+          ex.rk = p.round_key; ex.row = row_ptr<DT>(p, s.row); ex.tau = ri.tau; ex.grow = p.row_base + (uint32_t)s.row;
+          ex.ctr_lo = p.ctr_lo; ex.ctr_hi8 = p.ctr_hi8; ex.seg = 0; ex.V = (int)p.V;
+          id = sample_in_blocks<DT>(ex, top, lane, zt);
+          have_zt = id >= 0;
+        } else {
+          zt = pc.zf;
+          have_zt = id >= 0;
         }
-        EvalCtx ex;
-        ex.rk = p.round_key; ex.row = row_ptr<DT>(p, s.row); ex.tau = ri.tau; ex.grow = p.row_base + (uint32_t)s.row;
-        ex.ctr_lo = p.ctr_lo; ex.ctr_hi8 = p.ctr_hi8; ex.seg = 0; ex.V = (int)p.V;
-        id = sample_in_blocks<DT>(ex, top, lane);
       }
-      if (lane == 0) finish_row<DT>(p, s.row, ri, Md, Zd, Wd, yd, id, ed);
+      if (lane == 0) finish_row(p, s.row, ri, pc.M, pc.Z, pc.W, id, pc.err, have_zt, zt);
     }
   }
 }
@@ -1356,6 +1678,11 @@ struct KernelSetup {
 };
 
 template <int DT, int SAMPLER, bool RING>
+constexpr size_t dyn_smem_bytes() {
+  return (RING ? (size_t)kStages * kStageBytes : 0) + (SAMPLER == 0 ? (size_t)kStreamWarps * Fmt<DT>::kQueueBytes : 0);
+}
+
+template <int DT, int SAMPLER, bool RING>
 cudaError_t setup_kernel(KernelSetup &out) {
   static std::mutex lock;
   static KernelSetup cache[64];
@@ -1366,7 +1693,7 @@ cudaError_t setup_kernel(KernelSetup &out) {
   std::lock_guard<std::mutex> hold(lock);
   if (cache[dev].ctas_per_sm == 0) {
     auto kern = rows_kernel<DT, SAMPLER, RING>;
-    const size_t dyn = RING ? (size_t)kStages * kStageBytes : 0;
+    const size_t dyn = dyn_smem_bytes<DT, SAMPLER, RING>();
     e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn);
     if (e != cudaSuccess) return e;
     KernelSetup ks;
@@ -1397,27 +1724,22 @@ cudaError_t launch_one(RowsParams p, void *workspace, size_t workspace_bytes, cu
   if (slots > kMaxGrid) slots = kMaxGrid;
   p.tiles_per_row = (p.V + kTile - 1) / kTile;
   const int64_t tiles = p.rows * p.tiles_per_row;
+  p.narrow = tiles < (int64_t(1) << 31) ? 1 : 0;
   const bool can_cut = workspace != nullptr && workspace_bytes >= rows_workspace_bytes();
   // With a response mask the cost of a row is not known on the host: spread whole rows round-robin.
   p.interleaved = (!can_cut || (p.mask != nullptr && p.rows >= 4 * slots)) ? 1 : 0;
   int64_t grid = p.interleaved ? (p.rows < slots ? p.rows : slots) : (tiles < slots ? tiles : slots);
   p.tiles_q = tiles / grid;
   p.tiles_r = tiles % grid;
-  p.ws_pieces = nullptr;
-  p.ws_arrivals = nullptr;
-  if (can_cut) {
-    p.ws_pieces = static_cast<unsigned char *>(workspace);
-    p.ws_arrivals = reinterpret_cast<unsigned long long *>(p.ws_pieces + (size_t)kMaxGrid * 2 * kPieceBytes);
-  }
+  p.ws_pieces = can_cut ? static_cast<unsigned char *>(workspace) : nullptr;
   p.call_id = next_call_id();
-  const size_t dyn = RING ? (size_t)kStages * kStageBytes : 0;
-  rows_kernel<DT, SAMPLER, RING><<<(unsigned)grid, kThreads, dyn, stream>>>(p);
+  rows_kernel<DT, SAMPLER, RING><<<(unsigned)grid, kThreads, dyn_smem_bytes<DT, SAMPLER, RING>(), stream>>>(p);
   return cudaGetLastError();
 }
 
 }  // namespace
 
-size_t rows_workspace_bytes() { return (size_t)kMaxGrid * (2 * kPieceBytes + sizeof(unsigned long long)); }
+size_t rows_workspace_bytes() { return (size_t)kMaxGrid * 2 * kPieceBytes; }
 
 cudaError_t launch_rows(RowsParams p, int dtype, int sampler, bool aligned, void *workspace, size_t workspace_bytes,
                         cudaStream_t stream) {

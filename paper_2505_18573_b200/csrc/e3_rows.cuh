@@ -11,10 +11,11 @@ constexpr int kStreamThreads = kStreamWarps * 32;   // 256
 constexpr int kThreads = kStreamThreads + 64;       // + one warp that issues bulk copies + one that finishes rows
 constexpr int kGroup = 16;                          // vocabulary entries per coarse Philox call
 constexpr int kTile = 512;                          // unit of the work split (entries); CTA ranges start on tile bounds
-constexpr int kStageBytes = 16384;                   // bytes per pipeline stage (one bulk copy)
-constexpr int kStages = 6;
+constexpr int kLaneBytes = 64;                      // bytes a consumer thread takes from one pipeline stage
+constexpr int kStageBytes = kStreamThreads * kLaneBytes;  // 16 KiB per pipeline stage (one bulk copy)
+constexpr int kStages = 4;
 constexpr int kMaxGrid = 1024;                      // CTAs the piece workspace is sized for
-constexpr size_t kPieceBytes = 64;                  // one partial row state in the workspace
+constexpr size_t kPieceBytes = 128;                 // one partial row state in the workspace
 
 enum RowsMode : int { kModeSample = 0, kModeTargets = 1 };
 
@@ -35,18 +36,18 @@ struct RowsParams {
   int mode;
   // work split
   int interleaved;          // 1: CTA b takes whole rows b, b + grid, ...; 0: contiguous tile ranges (rows may be cut)
+  int narrow;               // 1: every tile number fits in 31 bits (32-bit index arithmetic on the device)
   int64_t tiles_per_row;    // ceil(V / kTile)
   int64_t tiles_q, tiles_r; // total tiles = grid * tiles_q + tiles_r: CTA b starts at tile b*tiles_q + min(b, tiles_r)
-  // cut rows: pieces and arrival words in the caller's workspace
-  unsigned char *ws_pieces;          // [grid][2] pieces of kPieceBytes
-  unsigned long long *ws_arrivals;   // [grid] (call id << 16 | pieces arrived), for the row whose first tile CTA k holds
+  // cut rows: partial states in the caller's workspace
+  unsigned char *ws_pieces;          // [grid][2] pieces of kPieceBytes, every word tagged with the call id
   unsigned long long call_id;        // unique per call within the process (48 bits)
 };
 
 size_t rows_workspace_bytes();
 
-// Launches the streaming kernel.  sampler: -1 = none (targets given), 0 = per-token Gumbel-max.
-// workspace may be nullptr: rows are then never cut (whole rows per CTA).
+// Launches the streaming kernel.  sampler: -1 = none (targets given), 0 = per-token Gumbel-max,
+// 1 = blocked Gumbel-max.  workspace may be nullptr: rows are then never cut (whole rows per CTA).
 cudaError_t launch_rows(RowsParams p, int dtype, int sampler, bool aligned, void *workspace, size_t workspace_bytes,
                         cudaStream_t stream);
 
