@@ -56,8 +56,12 @@ typedef enum { E3_F32 = 0, E3_BF16 = 1 } e3_dtype;
  * resolution of their uniforms (2^-40 and 2^-32). */
 typedef enum {
   E3_SAMPLER_TOKEN = 0, /* one Gumbel per vocabulary entry: tok = argmax_i (z_i/tau + g_i) */
-  E3_SAMPLER_BLOCK = 1  /* one Gumbel per block of E3_SAMPLE_BLOCK consecutive entries applied to the
+  E3_SAMPLER_BLOCK = 1, /* one Gumbel per block of E3_SAMPLE_BLOCK consecutive entries applied to the
                            block's log-sum-exp, then inverse CDF inside the winning block */
+  E3_SAMPLER_TOKEN_AUDIT = 2 /* the draw of E3_SAMPLER_TOKEN, token for token, computed the slow way: the fast
+                           path's fp32 scores (good to about 2e-4) are trusted only when the leader is
+                           ahead by a margin a thousand times wider than needed, so most rows are settled by
+                           the fp64 path that normally only sees near-ties.  For validation. */
 } e3_sampler;
 #define E3_SAMPLE_BLOCK 256
 

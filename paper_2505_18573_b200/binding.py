@@ -17,7 +17,7 @@ LIB_PATH = os.path.join(_PKG, "libe3.so")
 
 E3_OK = 0
 E3_F32, E3_BF16 = 0, 1
-E3_SAMPLER_TOKEN, E3_SAMPLER_BLOCK = 0, 1
+E3_SAMPLER_TOKEN, E3_SAMPLER_BLOCK, E3_SAMPLER_TOKEN_AUDIT = 0, 1, 2
 E3_CALL_SAMPLE, E3_CALL_TOKEN_LOGP_ENTROPY, E3_CALL_MASKED_MEAN_ENTROPY = 0, 1, 2
 E3_SAMPLE_BLOCK = 256
 

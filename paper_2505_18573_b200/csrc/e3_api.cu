@@ -53,7 +53,8 @@ extern "C" e3_status e3_sample(const void *logits, e3_dtype dt, int64_t rows, in
   e3_status st = check_logits(logits, dt, rows, V, row_stride);
   if (st != E3_OK) return st;
   if (misaligned(workspace, 16)) return E3_ERR_ALIGNMENT;
-  if (sampler != E3_SAMPLER_TOKEN && sampler != E3_SAMPLER_BLOCK) return E3_ERR_INVALID_ARG;
+  if (sampler != E3_SAMPLER_TOKEN && sampler != E3_SAMPLER_BLOCK && sampler != E3_SAMPLER_TOKEN_AUDIT)
+    return E3_ERR_INVALID_ARG;
   if (row_base < 0 || counter >= (uint64_t(1) << 56)) return E3_ERR_INVALID_ARG;
   if (rows == 0) return E3_OK;
   if (!temps || !out_tok) return E3_ERR_INVALID_ARG;
@@ -69,7 +70,8 @@ extern "C" e3_status e3_sample(const void *logits, e3_dtype dt, int64_t rows, in
   p.ctr_hi8 = static_cast<uint32_t>(counter >> 32) << 8;
   p.row_base = static_cast<uint32_t>(row_base);
   p.mode = e3::kModeSample;
-  cudaError_t e = e3::launch_rows(p, static_cast<int>(dt), static_cast<int>(sampler),
+  p.slack_scale = sampler == E3_SAMPLER_TOKEN_AUDIT ? 1000.f : 1.f;
+  cudaError_t e = e3::launch_rows(p, static_cast<int>(dt), sampler == E3_SAMPLER_BLOCK ? 1 : 0,
                                   rows_are_16B_aligned(logits, dt, row_stride), workspace, workspace_bytes,
                                   static_cast<cudaStream_t>(stream));
   return e == cudaSuccess ? E3_OK : E3_ERR_CUDA;
@@ -93,6 +95,7 @@ extern "C" e3_status e3_token_logp_entropy(const void *logits, e3_dtype dt, int6
   p.targets = targets; p.mask = mask;
   p.out_logp = out_logp; p.out_ent = out_ent;
   p.mode = e3::kModeTargets;
+  p.slack_scale = 1.f;
   cudaError_t e = e3::launch_rows(p, static_cast<int>(dt), -1, rows_are_16B_aligned(logits, dt, row_stride),
                                   workspace, workspace_bytes, static_cast<cudaStream_t>(stream));
   return e == cudaSuccess ? E3_OK : E3_ERR_CUDA;

@@ -91,26 +91,23 @@ struct Fmt {
 // the tag depends on the call and on the word, so a reader knows word by word whether what it sees was
 // written by this call (64-bit accesses are single-copy atomic); stale or half-written pieces fail the check.
 struct Piece {
-  double y;        // best perturbed score (greedy rows: largest logit)
   float M, Z, W;   // reference (log2 units), sum 2^t, sum 2^t t
-  int idx;         // vocabulary index of the best score, -1 = none
-  float zf;        // its logit
+  float zf;        // sampler 0: logit of entry tb[0]
   int err;
-  float ty[3];     // sampler 1: the three best block scores (fp32)
-  int tb[3];       // ... and their block indices, -1 = none
+  int pad;
+  float ty[3];     // the three best scores (fp32): sampler 0 entries, sampler 1 blocks; greedy rows: ty[0] = largest logit
+  int tb[3];       // ... and their vocabulary / block indices, -1 = none
 };
-constexpr int kPieceWords = 14;
+constexpr int kPieceWords = 12;
 static_assert(sizeof(Piece) == kPieceWords * 4, "piece payload");
 static_assert(kPieceWords * 8 <= kPieceBytes, "piece size");
 
 struct WarpPartial {
   float M, Z, W;
-  int idx;
-  double y;
+  float zf;
   int err;
   float ty[3];
   int tb[3];
-  float zf;
 };
 
 struct Smem {
@@ -147,14 +144,22 @@ struct AccS {
   float R, nRc, Z, W;
 };
 
+// Sampler 0: what a thread knows about the leaders of its row piece.  Scores are fp32 values of
+// y_i = z_i/tau + g_i, each within score_slack(y) of the exact value; the three best are kept so that
+// the finishing warp can tell whether fp32 separates the winner from the rest.  Greedy rows use
+// y[0] / b[0] for the largest logit and its index.
 struct Best {
-  double y;
-  int idx;
-  float zf;     // logit of entry idx
-  int enc;      // encoded lower bound of the row's best score known to this thread
+  float y[3];
+  int b[3];     // vocabulary indices, -1 = none; order: larger score first, equal scores by lower index
+  float zf;     // logit of entry b[0]
+  int enc;      // encoded value that is below the row's best score by at least four slacks
   float zthr;   // logit above which an entry may win whatever its coarse byte
   float zthr2;  // logit above which an entry with coarse byte 255 may win
 };
+// Bound on |fp32 score - exact score|: rounding of 1/tau, of the fused product-sum, of the integer
+// conversions and of the two approximate logarithms (worst for coarse byte 254: 1.1e-4).
+// k = 1 in normal operation; the audit sampler passes a large k, which sends most rows to the exact path.
+__device__ __forceinline__ float score_slack(float y, float k) { return k * (1.7e-4f + 1e-6f * fabsf(y)); }
 
 // ---------------------------------------------------------------------------------------------
 // small helpers
@@ -494,45 +499,62 @@ __device__ __forceinline__ float gate_threshold(int enc, float nRc) {
 struct EvalCtx {
   const uint32_t *rk;
   const char *row;
-  float tau;
+  float tau, slack_k;
   uint32_t grow, ctr_lo, ctr_hi8, seg;
   int V;
 };
 
-// One entry with logit zf and coarse byte cbyte: screen with an fp32 upper bound, then evaluate in fp64.
-__device__ __noinline__ void eval_element(const EvalCtx &x, int i, uint32_t cbyte, float zf, Best &b, Smem &sm) {
+// y_i = z_i/tau + g_i of the definition, in fp64 and in its expression order:
+// u = (c + (x + 1/2) 2^-32) / 256 (exact), g = -ln(-ln u).
+__device__ __noinline__ double exact_score(float zf, float tau, uint32_t cbyte, uint32_t xw) {
+  const double u = ((double)cbyte + ((double)xw + 0.5) * 0x1p-32) / 256.0;
+  const double s = (double)zf / (double)tau;
+  return s + (-log(-log(u)));
+}
+
+// fp32 value of y_i for fine word xw, coarse byte cbyte (within score_slack of the exact value).
+__device__ __forceinline__ float score_f32(float zf, float inv_tau, uint32_t cbyte, uint32_t xw) {
+  float w;  // -ln u
+  if (cbyte == 255u) {
+    // 1 - u = (2^32 - x - 1/2) 2^-40 < 2^-8 and -ln u = d + d^2/2 + d^3/3 + ...
+    const float d = ((float)(~xw) + 0.5f) * 0x1p-40f;
+    w = d * fmaf(d, fmaf(d, 0.33333334f, 0.5f), 1.0f);
+  } else {
+    const float u = ((float)cbyte + ((float)xw + 0.5f) * 0x1p-32f) * 0.00390625f;
+    w = -lg2f(u) * kLn2f;
+  }
+  return fmaf(zf, inv_tau, -lg2f(w) * kLn2f);
+}
+
+__device__ __forceinline__ bool best_before(float y, int i, float y2, int i2) {
+  return i2 < 0 || y > y2 || (y == y2 && i < i2);
+}
+// One entry with logit zf and coarse byte cbyte: cheap bounds first, then its fp32 score.
+__device__ __forceinline__ void consider(const uint32_t *rk, uint32_t grow, uint32_t ctr_lo, uint32_t ctr_hi8, float tau,
+                                         float inv_tau, float slack_k, uint32_t seg, int i, uint32_t cbyte, float zf,
+                                         Best &b, Smem &sm) {
   if (!(zf > b.zthr2) || zf == CUDART_INF_F) return;  // cannot win even with the largest Gumbel (also NaN, -inf)
   if (cbyte != 255u && !(zf > b.zthr)) return;
-  const uint4 fw = philox(x.rk, (uint32_t)i >> 2, x.grow, x.ctr_lo, x.ctr_hi8 | 1u);
-  const uint32_t xw = pick_word(fw, i & 3);
-  {
-    float gh;
-    if (cbyte == 255u) {
-      // 1 - u >= (2^32 - 1 - x) 2^-40 (and >= 2^-41); -ln u >= 1 - u, so g <= -ln(1 - u)
-      const float d = fmaxf((float)(~xw), 0.5f) * (0x1p-40f * 0.999999f);
-      gh = -lg2f(d) * kLn2f;
-    } else {
-      const float uh = fminf(((float)cbyte + ((float)xw + 1.0f) * 0x1p-32f) * (0.00390625f * 1.000001f), 0.9999f);
-      gh = -lg2f(-lg2f(uh) * kLn2f) * kLn2f;
-    }
-    const float sf = zf / x.tau;
-    const float yh = sf + fabsf(sf) * 2e-6f + gh + 2e-3f;
-    if (yh < dec_float(b.enc)) return;
-  }
-  // u = (c + (x + 1/2) 2^-32) / 256, exact in fp64; y = z/tau + (-ln(-ln u))
-  const double u = ((double)cbyte + ((double)xw + 0.5) * 0x1p-32) / 256.0;
-  const double s = (double)zf / (double)x.tau;
-  const double y = s + (-log(-log(u)));
-  if (y > b.y || (y == b.y && i < b.idx)) {
-    b.y = y;
-    b.idx = i;
+  const uint4 fw = philox(rk, (uint32_t)i >> 2, grow, ctr_lo, ctr_hi8 | 1u);
+  const float y = score_f32(zf, inv_tau, cbyte, pick_word(fw, i & 3));
+  if (!(y >= dec_float(b.enc))) return;  // more than two slacks below a score already seen (or NaN)
+  if (best_before(y, i, b.y[0], b.b[0])) {
+    b.y[2] = b.y[1]; b.b[2] = b.b[1]; b.y[1] = b.y[0]; b.b[1] = b.b[0]; b.y[0] = y; b.b[0] = i;
     b.zf = zf;
-    const int enc = enc_float(__double2float_rd(y));
+    const int enc = enc_float(y - 4.f * score_slack(y, slack_k) - 2e-7f * fabsf(y));
     if (enc > b.enc) {
-      set_gate(b, enc, x.tau);
-      post_best(sm, x.seg, enc);
+      set_gate(b, enc, tau);
+      post_best(sm, seg, enc);
     }
+  } else if (best_before(y, i, b.y[1], b.b[1])) {
+    b.y[2] = b.y[1]; b.b[2] = b.b[1]; b.y[1] = y; b.b[1] = i;
+  } else if (best_before(y, i, b.y[2], b.b[2])) {
+    b.y[2] = y; b.b[2] = i;
   }
+}
+
+__device__ __noinline__ void eval_element(const EvalCtx &x, int i, uint32_t cbyte, float zf, Best &b, Smem &sm) {
+  consider(x.rk, x.grow, x.ctr_lo, x.ctr_hi8, x.tau, __frcp_rn(x.tau), x.slack_k, x.seg, i, cbyte, zf, b, sm);
 }
 
 // A queue entry holds one group: 16 coarse bytes, then its 16 logits in vocabulary order.  Its header
@@ -543,40 +565,45 @@ __device__ __forceinline__ float entry_logit(const unsigned char *entry, int k) 
   return __uint_as_float((uint32_t)(*reinterpret_cast<const unsigned short *>(entry + 16 + 2 * k)) << 16);
 }
 
+// Evaluates the warp's queued groups, one per lane and round.  Everything it needs comes in registers
+// or from the queue in shared memory; only the rare fp64 evaluation is a call.
 template <int DT>
-__device__ __forceinline__ void eval_entry(const EvalCtx &x, const unsigned char *entry, int hdr, Best &b, Smem &sm) {
-  const int base = hdr & ~15;
-  const uint4 cw = *reinterpret_cast<const uint4 *>(entry);
-  uint32_t todo = 0;
-  {
-    const uint32_t w[4] = {cw.x, cw.y, cw.z, cw.w};
+__device__ __noinline__ void drain_queue(const uint32_t *rk, uint32_t grow, uint32_t ctr_lo, uint32_t ctr_hi8, float tau,
+                                         float slack_k, uint32_t seg, const unsigned char *queue, int qn, Best &best_io,
+                                         Smem &sm) {
+  const int lane = threadIdx.x & 31;
+  Best b = best_io;
+  const float inv_tau = __frcp_rn(tau);
+  __syncwarp();
+  const int *hdrs = reinterpret_cast<const int *>(queue);
+#pragma unroll 1
+  for (int e = lane; e < qn; e += 32) {
+    const unsigned char *entry = queue + kQueueHdrBytes + e * Fmt<DT>::kEntryBytes;
+    const int hdr = hdrs[e];
+    const uint4 cw = *reinterpret_cast<const uint4 *>(entry);
+    // bit k of todo: entry k of the group needs a look (its coarse byte is 255, or its logit is above the gate)
+    uint32_t todo = 0;
+    {
+      const uint32_t w[4] = {cw.x, cw.y, cw.z, cw.w};
 #pragma unroll
-    for (int q = 0; q < 4; ++q) {
-      const uint32_t m = ff_bytes(w[q]);
-      todo |= (((m >> 7) & 1u) | ((m >> 14) & 2u) | ((m >> 21) & 4u) | ((m >> 28) & 8u)) << (4 * q);
+      for (int q = 0; q < 4; ++q)  // bits 7, 15, 23, 31 -> one nibble
+        todo |= (((ff_bytes(w[q]) >> 7) * 0x10204080u) >> 28) << (4 * q);
+    }
+    if (hdr & 1) {
+#pragma unroll 1
+      for (int k = 0; k < 16; ++k)
+        if (entry_logit<DT>(entry, k) > b.zthr) todo |= 1u << k;
+    }
+#pragma unroll 1
+    while (todo) {
+      const int k = __ffs(todo) - 1;
+      todo &= todo - 1;
+      consider(rk, grow, ctr_lo, ctr_hi8, tau, inv_tau, slack_k, seg, (hdr & ~15) + k, entry[k], entry_logit<DT>(entry, k), b,
+               sm);
     }
   }
-  if (hdr & 1) {
-#pragma unroll 1
-    for (int k = 0; k < 16; ++k)
-      if (entry_logit<DT>(entry, k) > b.zthr) todo |= 1u << k;
-  }
-  while (todo) {
-    const int k = __ffs(todo) - 1;
-    todo &= todo - 1;
-    eval_element(x, base + k, entry[k], entry_logit<DT>(entry, k), b, sm);
-  }
-}
-
-// Evaluates the warp's queued groups, one per lane and round.
-template <int DT>
-__device__ __noinline__ void drain_queue(const EvalCtx &x, Best &b, Smem &sm, const unsigned char *queue, int qn) {
-  const int lane = threadIdx.x & 31;
   __syncwarp();
-  const int *hdr = reinterpret_cast<const int *>(queue);
-  for (int e = lane; e < qn; e += 32)
-    eval_entry<DT>(x, queue + kQueueHdrBytes + e * Fmt<DT>::kEntryBytes, hdr[e], b, sm);
-  __syncwarp();
+  best_io = b;
 }
 
 // Direct evaluation of one group held as floats (paths that do not stream from the ring).
@@ -800,10 +827,9 @@ __device__ __noinline__ void greedy_groups(SlowIO &io, const char *row, const un
       if (z[k] != z[k] || z[k] == CUDART_INF_F) io.err |= kErrValue;
       if (z[k] == gmax) kk = k;
     }
-    if (kk >= 0 && gmax > -CUDART_INF_F && (double)gmax > io.best.y) {
-      io.best.y = (double)gmax;
-      io.best.idx = g0 + kk;
-      io.best.zf = gmax;
+    if (kk >= 0 && gmax > -CUDART_INF_F && (io.best.b[0] < 0 || gmax > io.best.y[0])) {
+      io.best.y[0] = gmax;
+      io.best.b[0] = g0 + kk;
     }
   }
 }
@@ -840,7 +866,7 @@ __device__ __noinline__ void seed_piece(SeedIO &io, const EvalCtx &x, const unsi
       const float neg_ln_u = (8.0f - lg2f((float)cbyte + 0x1p-33f)) * kLn2f;
       const float glo = -lg2f(neg_ln_u) * kLn2f;
       const float sf = gmax / x.tau;
-      ylo = sf - fabsf(sf) * 2e-6f + glo - 2e-3f;
+      ylo = sf - fabsf(sf) * 8e-6f + glo - 4e-3f;  // also five score slacks below the entry's score
     }
     int enc = __reduce_max_sync(0xffffffffu, enc_float(ylo));
     if ((threadIdx.x & 31) == 0 && enc > enc_neg_inf()) post_best(sm, x.seg, enc);
@@ -865,14 +891,6 @@ __device__ __forceinline__ void merge_stats_f(float &M, float &Z, float &W, floa
   W = a * fmaf(d1, Z, W) + b * fmaf(d2, Z2, W2);
   Z = a * Z + b * Z2;
   M = Mn;
-}
-
-__device__ __forceinline__ void merge_best(double &y, int &idx, float &zf, double y2, int idx2, float zf2) {
-  if (idx2 >= 0 && (idx < 0 || y2 > y || (y2 == y && idx2 < idx))) {
-    y = y2;
-    idx = idx2;
-    zf = zf2;
-  }
 }
 
 __device__ __forceinline__ uint32_t piece_tag(u64 call_id, int j) {
@@ -905,11 +923,11 @@ __device__ __forceinline__ bool piece_load(const u64 *src, u64 call_id, Piece &p
 }
 
 // Merges the partial states held by the 32 lanes of a warp; every lane ends with the result.  A lane
-// without weight (Z = 0), without candidate (idx < 0) or with an empty list takes no part.  Written with
-// warp-wide reductions so that the chain of dependent instructions stays short: this runs at the end
-// of every row piece, when nothing else can hide it.  The order of all sums is fixed by lane numbers.
-template <int SAMPLER>
-__device__ __forceinline__ void warp_merge(Piece &pc, Top3 &top, bool with_best) {
+// without weight (Z = 0) or with an empty list takes no part.  Written with warp-wide reductions so
+// that the chain of dependent instructions stays short: this runs at the end of every row piece, when
+// nothing else can hide it.  The order of all sums is fixed by lane numbers.  with_top: the lists of
+// leaders (sampler 0 entries, sampler 1 blocks, greedy maxima) are merged too; pc.zf follows top.b[0].
+__device__ __forceinline__ void warp_merge(Piece &pc, Top3 &top, bool with_top) {
   constexpr unsigned kAll = 0xffffffffu;
   // softmax sums: move every lane to the largest reference, then add
   const bool has = pc.Z > 0.f;
@@ -930,29 +948,8 @@ __device__ __forceinline__ void warp_merge(Piece &pc, Top3 &top, bool with_best)
   }
   pc.M = Mw; pc.Z = Zs; pc.W = Ws;
   pc.err = __reduce_or_sync(kAll, pc.err);
-  if (with_best) {
-    // largest y, then lowest index: order-preserving 64-bit code of y, compared half by half
-    const long long bits = __double_as_longlong(pc.y);
-    const long long code = bits >= 0 ? bits : (bits ^ 0x7FFFFFFFFFFFFFFFll);
-    bool cand = pc.idx >= 0;
-    const int hi = cand ? (int)(code >> 32) : INT_MIN;
-    const int hmax = __reduce_max_sync(kAll, hi);
-    if (hmax == INT_MIN) {
-      pc.idx = -1;
-    } else {
-      cand = cand && hi == hmax;
-      const unsigned lo = cand ? (unsigned)code : 0u;
-      const unsigned lmax = __reduce_max_sync(kAll, lo);
-      cand = cand && lo == lmax;
-      const int imin = __reduce_min_sync(kAll, cand ? pc.idx : INT_MAX);
-      const int src = __ffs(__ballot_sync(kAll, cand && pc.idx == imin)) - 1;
-      pc.y = __shfl_sync(kAll, pc.y, src);
-      pc.zf = __shfl_sync(kAll, pc.zf, src);
-      pc.idx = imin;
-    }
-  }
-  if (SAMPLER == 1) {
-    // three rounds of "take the best head": larger score first, equal scores by lower block index
+  if (with_top) {
+    // three rounds of "take the best head": larger score first, equal scores by lower index
     Top3 out;
     top3_reset(out);
     int pos = 0;
@@ -967,11 +964,36 @@ __device__ __forceinline__ void warp_merge(Piece &pc, Top3 &top, bool with_best)
         const int bmin = __reduce_min_sync(kAll, c2 ? hb : INT_MAX);
         out.y[r] = dec_float(emax);
         out.b[r] = bmin;
-        if (c2 && hb == bmin) ++pos;
+        const bool mine = c2 && hb == bmin;
+        if (r == 0) pc.zf = __shfl_sync(kAll, pc.zf, __ffs(__ballot_sync(kAll, mine)) - 1);
+        if (mine) ++pos;
       }
     }
     top = out;
   }
+}
+
+// Largest y over the lanes, then lowest index (lanes with idx < 0 take no part); all lanes get the winner.
+__device__ __forceinline__ void warp_argmax_double(double &y, int &idx, float &zf) {
+  constexpr unsigned kAll = 0xffffffffu;
+  const long long bits = __double_as_longlong(y);
+  const long long code = bits >= 0 ? bits : (bits ^ 0x7FFFFFFFFFFFFFFFll);  // order-preserving
+  bool cand = idx >= 0 && y == y;
+  const int hi = cand ? (int)(code >> 32) : INT_MIN;
+  const int hmax = __reduce_max_sync(kAll, hi);
+  if (hmax == INT_MIN) {
+    idx = -1;
+    return;
+  }
+  cand = cand && hi == hmax;
+  const unsigned lo = cand ? (unsigned)code : 0u;
+  const unsigned lmax = __reduce_max_sync(kAll, lo);
+  cand = cand && lo == lmax;
+  const int imin = __reduce_min_sync(kAll, cand ? idx : INT_MAX);
+  const int src = __ffs(__ballot_sync(kAll, cand && idx == imin)) - 1;
+  y = __shfl_sync(kAll, y, src);
+  zf = __shfl_sync(kAll, zf, src);
+  idx = imin;
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -1270,6 +1292,57 @@ __device__ __noinline__ int sample_in_blocks(const EvalCtx &x, const Top3 &top, 
 }
 
 // ---------------------------------------------------------------------------------------------
+// Sampler 0, finishing warp: the leaders of the row are closer than fp32 can tell apart.  Every entry
+// whose fp32 score is within slack2 of the best may be the true winner; they are evaluated in fp64.
+// With one or two such entries they are in `top`; with three, others may exist and the whole row is
+// looked at again (fp32 scores for all entries, fp64 for those near the top).
+// ---------------------------------------------------------------------------------------------
+template <int DT>
+__device__ __noinline__ int settle_exact(const EvalCtx &x, const Top3 &top, float slack2, int lane, float &z_tok) {
+  double ybest = -CUDART_INF;
+  int ibest = -1;
+  float zbest = 0.f;
+  const bool rescan = top.b[2] >= 0 && !(top.y[0] - top.y[2] > slack2);
+  if (!rescan) {
+    const int i = lane == 0 ? top.b[0] : (lane == 1 ? top.b[1] : -1);
+    if (i >= 0) {
+      const float z = load_elem<DT>(x.row, i);
+      const uint4 cw = philox(x.rk, (uint32_t)i >> 4, x.grow, x.ctr_lo, x.ctr_hi8 | 0u);
+      const uint32_t cbyte = (pick_word(cw, (i & 15) >> 2) >> (8 * (i & 3))) & 0xFFu;
+      const uint4 fw = philox(x.rk, (uint32_t)i >> 2, x.grow, x.ctr_lo, x.ctr_hi8 | 1u);
+      ybest = exact_score(z, x.tau, cbyte, pick_word(fw, i & 3));
+      ibest = i;
+      zbest = z;
+    }
+  } else {
+    const float inv_tau = __frcp_rn(x.tau);
+    const float floor_y = top.y[0] - slack2;
+#pragma unroll 1
+    for (int q0 = lane * 4; q0 < x.V; q0 += 128) {  // four entries (one fine call) per lane and round
+      const uint4 cw = philox(x.rk, (uint32_t)q0 >> 4, x.grow, x.ctr_lo, x.ctr_hi8 | 0u);
+      const uint32_t cword = pick_word(cw, (q0 & 15) >> 2);
+      const uint4 fw = philox(x.rk, (uint32_t)q0 >> 2, x.grow, x.ctr_lo, x.ctr_hi8 | 1u);
+#pragma unroll 1
+      for (int k = 0; k < 4 && q0 + k < x.V; ++k) {
+        const float z = load_elem<DT>(x.row, q0 + k);
+        if (!(z > -CUDART_INF_F && z < CUDART_INF_F)) continue;
+        const uint32_t cbyte = (cword >> (8 * k)) & 0xFFu, xw = pick_word(fw, k);
+        if (!(score_f32(z, inv_tau, cbyte, xw) >= floor_y)) continue;
+        const double y = exact_score(z, x.tau, cbyte, xw);
+        if (ibest < 0 || y > ybest) {  // indices ascend within a lane
+          ybest = y;
+          ibest = q0 + k;
+          zbest = z;
+        }
+      }
+    }
+  }
+  warp_argmax_double(ybest, ibest, zbest);
+  z_tok = zbest;
+  return ibest;
+}
+
+// ---------------------------------------------------------------------------------------------
 // The kernel
 // ---------------------------------------------------------------------------------------------
 template <int DT, int SAMPLER, bool RING>
@@ -1327,13 +1400,16 @@ __global__ void __launch_bounds__(kThreads, 2) rows_kernel(const __grid_constant
       const uint32_t seg = n + 1;
 #define E3_MAKE_CTX(ex)                                                                                  \
   EvalCtx ex;                                                                                            \
-  ex.rk = rk; ex.row = row; ex.tau = ri.tau; ex.grow = grow; ex.ctr_lo = p.ctr_lo; ex.ctr_hi8 = p.ctr_hi8; \
+  ex.rk = rk; ex.row = row; ex.tau = ri.tau; ex.slack_k = p.slack_scale; ex.grow = grow; ex.ctr_lo = p.ctr_lo; \
+  ex.ctr_hi8 = p.ctr_hi8;                                                                                \
   ex.seg = seg; ex.V = (int)p.V
 
       Acc acc;
       acc_reset(acc);
       Best best;
-      best.y = -CUDART_INF; best.idx = -1; best.zf = 0.f;
+      best.y[0] = best.y[1] = best.y[2] = -CUDART_INF_F;
+      best.b[0] = best.b[1] = best.b[2] = -1;
+      best.zf = 0.f;
       set_gate(best, enc_neg_inf(), ri.tau);
       float ethr = 0.f;
       int err = 0, qn = 0;
@@ -1448,8 +1524,7 @@ __global__ void __launch_bounds__(kThreads, 2) rows_kernel(const __grid_constant
                 qn += __popc(ballot);
                 if (qn >= kDrainAt) {
                   Best tb = best;
-                  E3_MAKE_CTX(ex);
-                  drain_queue<DT>(ex, tb, sm, queue, qn);
+                  drain_queue<DT>(rk, grow, p.ctr_lo, p.ctr_hi8, ri.tau, p.slack_scale, seg, queue, qn, tb, sm);
                   best = tb;
                   qn = 0;
                   const int enc = read_best(sm, seg);
@@ -1488,8 +1563,7 @@ __global__ void __launch_bounds__(kThreads, 2) rows_kernel(const __grid_constant
       }
       if (SAMPLER == 0 && qn > 0) {
         Best tb = best;
-        E3_MAKE_CTX(ex);
-        drain_queue<DT>(ex, tb, sm, queue, qn);
+        drain_queue<DT>(rk, grow, p.ctr_lo, p.ctr_hi8, ri.tau, p.slack_scale, seg, queue, qn, tb, sm);
         best = tb;
         qn = 0;
       }
@@ -1522,13 +1596,17 @@ __global__ void __launch_bounds__(kThreads, 2) rows_kernel(const __grid_constant
       Piece pw;
       pw.M = -fin.nRc; pw.Z = fin.Z; pw.W = fin.W;
       if (fin.R == -CUDART_INF_F) { pw.M = 0.f; pw.Z = 0.f; pw.W = 0.f; }
-      pw.y = best.y; pw.idx = best.idx; pw.zf = best.zf; pw.err = err;
-      warp_merge<SAMPLER>(pw, bs.top, p.mode == kModeSample);
+      pw.zf = best.zf; pw.err = err;
+      if (SAMPLER != 1 || ri.greedy) {  // sampler 0 and greedy rows: the thread's leaders; sampler 1: its blocks
+#pragma unroll
+        for (int i = 0; i < 3; ++i) { bs.top.y[i] = best.y[i]; bs.top.b[i] = best.b[i]; }
+      }
+      warp_merge(pw, bs.top, SAMPLER >= 0);
       const uint32_t slot = n % kSlots, use = n / kSlots;
       if (use > 0) mbar_wait(&sm.wfree[slot], (use - 1) & 1u, sm);
       if (lane == 0) {
         WarpPartial &w = sm.wpart[slot][warp];
-        w.M = pw.M; w.Z = pw.Z; w.W = pw.W; w.y = pw.y; w.idx = pw.idx; w.err = pw.err; w.zf = pw.zf;
+        w.M = pw.M; w.Z = pw.Z; w.W = pw.W; w.err = pw.err; w.zf = pw.zf;
 #pragma unroll
         for (int i = 0; i < 3; ++i) { w.ty[i] = bs.top.y[i]; w.tb[i] = bs.top.b[i]; }
         mbar_arrive(&sm.wfull[slot]);
@@ -1595,13 +1673,13 @@ __global__ void __launch_bounds__(kThreads, 2) rows_kernel(const __grid_constant
       const uint32_t slot = n % kSlots, use = n / kSlots;
       mbar_wait_warp(&sm.wfull[slot], use & 1u, sm, lane);
       Piece pc;
-      pc.y = -CUDART_INF; pc.M = 0.f; pc.Z = 0.f; pc.W = 0.f; pc.idx = -1; pc.zf = 0.f; pc.err = 0;
+      pc.M = 0.f; pc.Z = 0.f; pc.W = 0.f; pc.zf = 0.f; pc.err = 0; pc.pad = 0;
       Top3 top;
       top3_reset(top);
       if (lane < kStreamWarps) {
         const WarpPartial &w = sm.wpart[slot][lane];
-        pc.M = w.M; pc.Z = w.Z; pc.W = w.W; pc.y = w.y; pc.idx = w.idx; pc.err = w.err; pc.zf = w.zf;
-        if (SAMPLER == 1) {
+        pc.M = w.M; pc.Z = w.Z; pc.W = w.W; pc.err = w.err; pc.zf = w.zf;
+        if (SAMPLER >= 0) {
 #pragma unroll
           for (int i = 0; i < 3; ++i) { top.y[i] = w.ty[i]; top.b[i] = w.tb[i]; }
         }
@@ -1611,7 +1689,7 @@ __global__ void __launch_bounds__(kThreads, 2) rows_kernel(const __grid_constant
       ++n;
       // The order of every merge below is fixed by lane and piece numbers alone, so the result does not
       // depend on which CTA ends up finishing the row.
-      warp_merge<SAMPLER>(pc, top, sample);
+      warp_merge(pc, top, SAMPLER >= 0);
       if (*reinterpret_cast<volatile int *>(&sm.timeout)) pc.err |= kErrTimeout;
       bool fin = s.whole;
       if (!s.whole) {
@@ -1626,7 +1704,7 @@ __global__ void __launch_bounds__(kThreads, 2) rows_kernel(const __grid_constant
           asm volatile("fence.sc.gpu;" ::: "memory");
         }
         __syncwarp();
-        pc.y = -CUDART_INF; pc.M = 0.f; pc.Z = 0.f; pc.W = 0.f; pc.idx = -1; pc.zf = 0.f; pc.err = 0;
+        pc.M = 0.f; pc.Z = 0.f; pc.W = 0.f; pc.zf = 0.f; pc.err = 0;
         top3_reset(top);
         bool ok = true;
         for (int k = s.k0 + lane; k <= s.k1; k += 32) {
@@ -1639,28 +1717,34 @@ __global__ void __launch_bounds__(kThreads, 2) rows_kernel(const __grid_constant
           }
           pc.err |= q.err;
           merge_stats_f(pc.M, pc.Z, pc.W, q.M, q.Z, q.W);
-          merge_best(pc.y, pc.idx, pc.zf, q.y, q.idx, q.zf);
-          if (SAMPLER == 1) {
+          if (SAMPLER >= 0) {
+            if (q.tb[0] >= 0 && best_before(q.ty[0], q.tb[0], top.y[0], top.b[0])) pc.zf = q.zf;
 #pragma unroll
             for (int i = 0; i < 3; ++i) top3_insert(top, q.ty[i], q.tb[i]);
           }
         }
         fin = __all_sync(0xffffffffu, ok);
-        if (fin) warp_merge<SAMPLER>(pc, top, sample);
+        if (fin) warp_merge(pc, top, SAMPLER >= 0);
       }
       if (!fin) continue;
-      int id = pc.idx;
+      int id = -1;
       bool have_zt = !sample && target >= 0 && target < p.V;
-      if (sample && !ri.greedy) {
-        if (SAMPLER == 1) {
-          // the whole warp settles the block and draws inside it
+      if (SAMPLER >= 0) {
+        id = top.b[0];
+        if (!ri.greedy && id >= 0) {
           EvalCtx ex;
-          ex.rk = p.round_key; ex.row = row_ptr<DT>(p, s.row); ex.tau = ri.tau; ex.grow = p.row_base + (uint32_t)s.row;
+          ex.rk = p.round_key; ex.row = row_ptr<DT>(p, s.row); ex.tau = ri.tau; ex.slack_k = p.slack_scale;
+          ex.grow = p.row_base + (uint32_t)s.row;
           ex.ctr_lo = p.ctr_lo; ex.ctr_hi8 = p.ctr_hi8; ex.seg = 0; ex.V = (int)p.V;
-          id = sample_in_blocks<DT>(ex, top, lane, zt);
-          have_zt = id >= 0;
-        } else {
-          zt = pc.zf;
+          if (SAMPLER == 1) {
+            // the whole warp settles the block and draws inside it
+            id = sample_in_blocks<DT>(ex, top, lane, zt);
+          } else {
+            // fp32 scores decide unless the runner-up is within two slacks of the leader
+            zt = pc.zf;
+            const float slack2 = 2.f * fmaxf(score_slack(top.y[0], p.slack_scale), score_slack(top.y[1], p.slack_scale));
+            if (top.b[1] >= 0 && !(top.y[0] - top.y[1] > slack2)) id = settle_exact<DT>(ex, top, slack2, lane, zt);
+          }
           have_zt = id >= 0;
         }
       }

@@ -34,6 +34,7 @@ struct RowsParams {
   uint32_t ctr_hi8;         // (high bits of the step counter) << 8; the stream tag is OR-ed in
   uint32_t row_base;
   int mode;
+  float slack_scale;        // 1; the audit sampler widens the fp32 score slack so that rows are settled in fp64
   // work split
   int interleaved;          // 1: CTA b takes whole rows b, b + grid, ...; 0: contiguous tile ranges (rows may be cut)
   int narrow;               // 1: every tile number fits in 31 bits (32-bit index arithmetic on the device)
@@ -47,7 +48,7 @@ struct RowsParams {
 size_t rows_workspace_bytes();
 
 // Launches the streaming kernel.  sampler: -1 = none (targets given), 0 = per-token Gumbel-max,
-// 1 = blocked Gumbel-max.  workspace may be nullptr: rows are then never cut (whole rows per CTA).
+// 1 = blocked Gumbel-max (the caller sets slack_scale).  workspace may be nullptr: rows are then never cut (whole rows per CTA).
 cudaError_t launch_rows(RowsParams p, int dtype, int sampler, bool aligned, void *workspace, size_t workspace_bytes,
                         cudaStream_t stream);
 

@@ -125,6 +125,31 @@ def test_padded_stride_and_unaligned_rows(e3, dtype):
         _check_sample(e3, odd[:, 1:V + 1], temps, seed=1, counter=4, sampler=sampler, name="offset1")
 
 
+def test_audit_sampler_settles_rows_in_fp64_and_agrees(e3):
+    """E3_SAMPLER_TOKEN_AUDIT distrusts the fp32 scores of the fast path (slack x 1000), so rows whose two or
+    three leaders lie within ~0.35 of each other are settled by the fp64 path (two contenders) or by the
+    second look at the whole row (three or more): both must give the token of the definition."""
+    for rows, V, dtype, seed in ((256, 4000, torch.float32, 90), (64, 151936, torch.bfloat16, 91),
+                                 (40, 33333, torch.bfloat16, 92), (300, 129, torch.float32, 93)):
+        logits = inputs.zipf_gaussian_logits(rows, V, seed=seed, dtype=dtype, device=DEV)
+        temps = inputs.uniform_temps(rows, seed=seed + 1, device=DEV)
+        ref = oracle.sample(inputs.to_oracle_array(logits), temps.cpu().numpy(), 7, seed, 0, 0)
+        gap = ref.y1 - ref.y2
+        assert (gap < 0.3).sum() >= 5, "the case must contain rows that take the exact path"
+        tok, lp, en = _run_sample(e3, logits, temps, 7, seed, 0, e3.E3_SAMPLER_TOKEN_AUDIT)
+        fast, lp0, en0 = _run_sample(e3, logits, temps, 7, seed, 0, e3.E3_SAMPLER_TOKEN)
+        assert_tokens("audit", tok, ref, 0)
+        assert np.array_equal(tok, fast)
+        assert_close("audit.logp", lp, ref.logp, ATOL[dtype])
+        assert_close("audit.ent", en, ref.ent, ATOL[dtype])
+    # flat rows: many entries within the widened slack of the leader
+    logits = inputs.onehot_flat_logits(16, 256000, seed=94, device=DEV)
+    temps = inputs.loguniform_temps(16, seed=95, device=DEV)
+    ref = oracle.sample(logits.cpu().numpy(), temps.cpu().numpy(), 1, 2, 0, 0)
+    tok, lp, en = _run_sample(e3, logits, temps, 1, 2, 0, e3.E3_SAMPLER_TOKEN_AUDIT)
+    assert_tokens("audit.flat", tok, ref, 0)
+
+
 def test_empty_batch_is_a_noop(e3):
     logits = torch.zeros((0, 100), dtype=torch.float32, device=DEV)
     tok, lp, en = e3.e3_sample(logits, torch.zeros(0, device=DEV), 0, 0)
