@@ -54,6 +54,7 @@ namespace e3 {
 namespace {
 
 using u64 = unsigned long long;
+using f2 = float2;  // two fp32 values in a register pair
 
 constexpr int kQueueCap = 64;   // candidate groups a warp can hold
 constexpr int kDrainAt = 32;    // ... and the fill at which it evaluates them (one per lane)
@@ -137,7 +138,7 @@ struct Seg {
 // Running sums of a consumer thread, two fp32 lanes per register pair.
 struct Acc {
   float R, nRc;      // reference logit and -R*c; R = -inf, nRc = kNoRef: no reference yet
-  u64 Z2, Wa2, Wb2;  // Z = sum of both halves of Z2, W = sum of the four halves of Wa2, Wb2
+  f2 Z2, Wa2, Wb2;   // Z = sum of both halves of Z2, W = sum of the four halves of Wa2, Wb2
 };
 // The same state as plain scalars (careful form).
 struct AccS {
@@ -174,34 +175,11 @@ __device__ __forceinline__ float lg2f(float x) {
   asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
-__device__ __forceinline__ u64 pack2(uint32_t lo, uint32_t hi) {
-  u64 d;
-  asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "r"(lo), "r"(hi));
-  return d;
-}
-__device__ __forceinline__ u64 pack2f(float lo, float hi) { return pack2(__float_as_uint(lo), __float_as_uint(hi)); }
-__device__ __forceinline__ void unpack2(u64 v, float &lo, float &hi) {
-  uint32_t a, b;
-  asm("mov.b64 {%0, %1}, %2;" : "=r"(a), "=r"(b) : "l"(v));
-  lo = __uint_as_float(a);
-  hi = __uint_as_float(b);
-}
-__device__ __forceinline__ float sum2(u64 v) {
-  float a, b;
-  unpack2(v, a, b);
-  return a + b;
-}
-// Packed fp32 arithmetic: both halves of a 64-bit register pair in one instruction.
-__device__ __forceinline__ u64 fma2(u64 a, u64 b, u64 c) {
-  u64 d;
-  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
-  return d;
-}
-__device__ __forceinline__ u64 add2(u64 a, u64 b) {
-  u64 d;
-  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
-  return d;
-}
+// Packed fp32 arithmetic: both halves of a register pair in one instruction.
+__device__ __forceinline__ f2 pack2f(float lo, float hi) { return make_float2(lo, hi); }
+__device__ __forceinline__ float sum2(f2 v) { return v.x + v.y; }
+__device__ __forceinline__ f2 fma2(f2 a, f2 b, f2 c) { return __ffma2_rn(a, b, c); }
+__device__ __forceinline__ f2 add2(f2 a, f2 b) { return __fadd2_rn(a, b); }
 // max that keeps NaN (a NaN logit must reach the sums)
 __device__ __forceinline__ uint32_t floor_bf16x2(uint32_t w) {
   uint32_t d;
@@ -363,7 +341,7 @@ constexpr float kNoRef = 1e30f;  // nRc of a state without reference: the first 
 __device__ __forceinline__ void acc_reset(Acc &a) {
   a.R = -CUDART_INF_F;
   a.nRc = kNoRef;
-  a.Z2 = a.Wa2 = a.Wb2 = 0ull;
+  a.Z2 = a.Wa2 = a.Wb2 = pack2f(0.f, 0.f);
 }
 __device__ __forceinline__ AccS to_scalar(const Acc &a) {
   AccS s;
@@ -378,7 +356,7 @@ __device__ __forceinline__ void from_scalar(Acc &a, const AccS &s) {
   a.nRc = s.nRc;
   a.Z2 = pack2f(s.Z, 0.f);
   a.Wa2 = pack2f(s.W, 0.f);
-  a.Wb2 = 0ull;
+  a.Wb2 = pack2f(0.f, 0.f);
 }
 
 // Careful form for one group: accepts any values.  -inf entries carry no weight, NaN and +inf flag the
@@ -428,43 +406,28 @@ __device__ __forceinline__ float careful_accumulate(AccS &a, const float (&z)[16
 // Streaming form for one group held in raw 16-byte vectors (any order): adds sum 2^t t to (Wa2, Wb2),
 // returns the packed group sum of 2^t in Zg2 and its scalar value.
 template <int DT>
-__device__ __forceinline__ float hot_group(const uint4 *v, u64 c2, u64 nRc2, u64 &Wa2, u64 &Wb2, u64 &Zg2) {
-  u64 Za = 0ull, Zb = 0ull;
+__device__ __forceinline__ float hot_group(const uint4 *v, f2 c2, f2 nRc2, f2 &Wa2, f2 &Wb2, f2 &Zg2) {
+  f2 Za = pack2f(0.f, 0.f), Zb = pack2f(0.f, 0.f);
 #pragma unroll
   for (int q = 0; q < Fmt<DT>::kVG; ++q) {
     const uint32_t w[4] = {v[q].x, v[q].y, v[q].z, v[q].w};
-    if (DT == 1) {
 #pragma unroll
-      for (int j = 0; j < 4; ++j) {
+    for (int j = 0; j < (DT == 1 ? 4 : 2); ++j) {
+      f2 z2;
+      if (DT == 1) {
         const uint32_t x = floor_bf16x2(w[j]);
-        const u64 z2 = pack2(x << 16, x & 0xFFFF0000u);
-        const u64 t2 = fma2(z2, c2, nRc2);
-        float tl, th;
-        unpack2(t2, tl, th);
-        const u64 e2 = pack2f(ex2f(tl), ex2f(th));
-        if (j & 1) {
-          Zb = (q == 0 && j == 1) ? e2 : add2(Zb, e2);
-          Wb2 = fma2(e2, t2, Wb2);
-        } else {
-          Za = (q == 0 && j == 0) ? e2 : add2(Za, e2);
-          Wa2 = fma2(e2, t2, Wa2);
-        }
+        z2 = pack2f(__uint_as_float(x << 16), __uint_as_float(x & 0xFFFF0000u));
+      } else {
+        z2 = pack2f(__uint_as_float(floor_f32(w[2 * j])), __uint_as_float(floor_f32(w[2 * j + 1])));
       }
-    } else {
-#pragma unroll
-      for (int j = 0; j < 2; ++j) {
-        const u64 z2 = pack2(floor_f32(w[2 * j]), floor_f32(w[2 * j + 1]));
-        const u64 t2 = fma2(z2, c2, nRc2);
-        float tl, th;
-        unpack2(t2, tl, th);
-        const u64 e2 = pack2f(ex2f(tl), ex2f(th));
-        if (j & 1) {
-          Zb = (q == 0) ? e2 : add2(Zb, e2);
-          Wb2 = fma2(e2, t2, Wb2);
-        } else {
-          Za = (q == 0) ? e2 : add2(Za, e2);
-          Wa2 = fma2(e2, t2, Wa2);
-        }
+      const f2 t2 = fma2(z2, c2, nRc2);
+      const f2 e2 = pack2f(ex2f(t2.x), ex2f(t2.y));
+      if (j & 1) {
+        Zb = add2(Zb, e2);
+        Wb2 = fma2(e2, t2, Wb2);
+      } else {
+        Za = add2(Za, e2);
+        Wa2 = fma2(e2, t2, Wa2);
       }
     }
   }
@@ -1474,7 +1437,7 @@ __global__ void __launch_bounds__(kThreads, 2) rows_kernel(const __grid_constant
           // raw[kVG*gi ...] is group gi ^ ga of the thread (vocabulary order)
           const int ga = kG == 2 ? (rot >> 1) : 0;
           const Acc saved = acc;
-          const u64 c2 = pack2f(ri.c, ri.c), nRc2 = pack2f(acc.nRc, acc.nRc);
+          const f2 c2 = pack2f(ri.c, ri.c), nRc2 = pack2f(acc.nRc, acc.nRc);
           float Zg[kG];
           bool have[kG];
           bool bad = false;
@@ -1484,7 +1447,7 @@ __global__ void __launch_bounds__(kThreads, 2) rows_kernel(const __grid_constant
             have[gi] = g0 + kGroup <= lim;
             Zg[gi] = 0.f;
             if (have[gi]) {
-              u64 Zg2;
+              f2 Zg2;
               Zg[gi] = hot_group<DT>(&raw[kVG * gi], c2, nRc2, acc.Wa2, acc.Wb2, Zg2);
               acc.Z2 = add2(acc.Z2, Zg2);
               bad |= !(Zg[gi] <= kGroupSumMax);
