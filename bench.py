@@ -18,6 +18,10 @@ device and its tokens device -> host inside the timed region.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--sampler 0|1] [--impl e3|reference]
 
+The step uses sampler 1 (blocked Gumbel-max) unless told otherwise; `kernels` in the output line
+gives the device time of every row kernel alone (both samplers and the training-side pass), timed
+with CUDA events over the same ring of logits.
+
 Under torchrun (N > 1) every rank runs the same per-GPU batch with its own row_base (weak
 scaling; rows are independent, the only exchange is a 16-byte all-reduce of the entropy sum
 and count).  `--impl reference` times the fp64 CPU oracle on a bounded sample of the same
@@ -170,7 +174,8 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--sampler", type=int, default=0, choices=[0, 1])
+    ap.add_argument("--sampler", type=int, default=1, choices=[0, 1],
+                    help="0 = one Gumbel per vocabulary entry, 1 = one Gumbel per block of 256 entries (default)")
     ap.add_argument("--impl", default="e3", choices=["e3", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -335,6 +340,29 @@ def main():
                "h2d_bytes_per_step": (DECODE_STEPS + RING) * ROWS * V * 2 + ROWS * 4,
                "d2h_bytes_per_step": DECODE_STEPS * ROWS * 4 + 16}
 
+    # ---- every row kernel alone (device time, CUDA events, same ring) -------------------------------
+    def time_alone(fn, reps=64):
+        for d in range(RING):
+            fn(d)
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for d in range(reps):
+            fn(d)
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) * 1e3 / reps
+
+    targets1 = all_toks[:ROWS]
+    alone = {
+        "e3_sample[sampler 0]": time_alone(lambda d: e3.e3_sample(ring[d % RING], temps, 0, d, row_base, 0,
+                                                                    out_tok=toks[d % RING], out_logp=logp, out_ent=ent)),
+        "e3_sample[sampler 1]": time_alone(lambda d: e3.e3_sample(ring[d % RING], temps, 0, d, row_base, 1,
+                                                                    out_tok=toks[d % RING], out_logp=logp, out_ent=ent)),
+        "e3_token_logp_entropy": time_alone(lambda d: e3.e3_token_logp_entropy(ring[d % RING], targets1, temps=temps,
+                                                                                 out_logp=logp, out_ent=ent)),
+    }
+
     if rank == 0:
         peak, peak_kind = _peaks()
         bytes_per_launch = ROWS * V * 2 + ROWS * 4 + ROWS * 12
@@ -350,11 +378,14 @@ def main():
                        "decode_steps": DECODE_STEPS, "l2": f"ring of {RING} logits buffers (1.24 GB) larger than L2",
                        "step": "256 x e3_sample + e3_token_logp_entropy(4096 rows) + masked mean + group advantage + host tau update",
                        "e2e_steps": args.e2e_steps},
-            "roofline": {"bound": "hbm", "kernel": "rows_kernel (e3_sample, bf16)", "achieved": achieved, "peak": peak,
+            "roofline": {"bound": "hbm", "kernel": f"rows_kernel (e3_sample, sampler {args.sampler}, bf16)",
+                         "achieved": achieved, "peak": peak,
                          "peak_kind": peak_kind, "unit": "GB/s", "frac": achieved / peak, "frac_of_8TBs": achieved / 8000.0,
                          "us_per_launch": launch_s * 1e6, "bytes_per_launch": bytes_per_launch, "traffic": None},
             "training_side": {"ms_per_step": ms_tail / args.steps, "unmasked_rows": unmasked,
                               "GBps_incl_small_kernels_and_sync": train_bytes / (ms_tail * 1e-3 / args.steps) / 1e9},
+            "kernels": {k: {"us_per_launch": v, "GBps": bytes_per_launch / v / 1e3, "frac": bytes_per_launch / v / 1e3 / peak}
+                        for k, v in alone.items()},
             "e2e": e2e,
             "gpu_launches": launches_per_step * args.steps,
             "clocks": clocks.summary(),
