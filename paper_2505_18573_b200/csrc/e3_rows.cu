@@ -68,8 +68,11 @@ constexpr double kLn2 = 0.6931471805599453094;
 // with all 40 bits set the largest value is -ln(-ln(1 - 2^-41)) = 28.41903...  Both rounded up.
 constexpr float kGumbelCapCoarse = 5.5433f;
 constexpr float kGumbelCapAll = 28.4192f;
-// A group whose sum of 2^t is above this (or NaN) leaves the streaming form: its reference is stale.
-constexpr float kGroupSumMax = 1.0995116e12f;  // 2^40
+// A group of 16 whose sum of 2^t is above this (or NaN) means that the warp's reference logit is stale:
+// the warp moves it up to the largest logit of the current turn and repeats the group.  Every entry that
+// is added therefore has t <= 5 while the reference is a logit the warp has really seen, so W/Z stays
+// small and the entropy ln Z - ln2 W/Z is free of cancellation at the 1e-5 level.
+constexpr float kGroupSumMax = 32.f;
 // Logits below this (also -inf) enter the streaming form as this value: weight 2^-huge = 0.
 constexpr uint32_t kFloorBf16x2 = 0xF180F180u;  // -2^100 twice
 constexpr float kFloorF32 = -1.2676506e30f;     // -2^100
@@ -180,6 +183,7 @@ __device__ __forceinline__ f2 pack2f(float lo, float hi) { return make_float2(lo
 __device__ __forceinline__ float sum2(f2 v) { return v.x + v.y; }
 __device__ __forceinline__ f2 fma2(f2 a, f2 b, f2 c) { return __ffma2_rn(a, b, c); }
 __device__ __forceinline__ f2 add2(f2 a, f2 b) { return __fadd2_rn(a, b); }
+__device__ __forceinline__ f2 mul2(f2 a, f2 b) { return __fmul2_rn(a, b); }
 // max that keeps NaN (a NaN logit must reach the sums)
 __device__ __forceinline__ uint32_t floor_bf16x2(uint32_t w) {
   uint32_t d;
@@ -401,6 +405,28 @@ __device__ __forceinline__ float careful_accumulate(AccS &a, const float (&z)[16
   }
   a.Z += g;
   return g;
+}
+
+// Largest logit of one group held in raw 16-byte vectors (NaN entries are passed over).
+template <int DT>
+__device__ __forceinline__ float group_max(const uint4 *v) {
+  if (DT == 1) {
+    uint32_t m = v[0].x;
+#pragma unroll
+    for (int q = 0; q < 2; ++q) {
+      const uint32_t w[4] = {v[q].x, v[q].y, v[q].z, v[q].w};
+#pragma unroll
+      for (int j = 0; j < 4; ++j) asm("max.bf16x2 %0, %1, %2;" : "=r"(m) : "r"(m), "r"(w[j]));
+    }
+    return fmaxf(__uint_as_float(m << 16), __uint_as_float(m & 0xFFFF0000u));
+  } else {
+    float m = -CUDART_INF_F;
+#pragma unroll
+    for (int q = 0; q < 4; ++q)
+      m = fmaxf(fmaxf(m, fmaxf(__uint_as_float(v[q].x), __uint_as_float(v[q].y))),
+                fmaxf(__uint_as_float(v[q].z), __uint_as_float(v[q].w)));
+    return m;
+  }
 }
 
 // Streaming form for one group held in raw 16-byte vectors (any order): adds sum 2^t t to (Wa2, Wb2),
@@ -973,40 +999,48 @@ __device__ __forceinline__ int cta_of_tile(const RowsParams &p, int64_t t) {
   return (int)(t < big ? quot(p, t, p.tiles_q + 1) : p.tiles_r + quot(p, t - big, p.tiles_q));
 }
 
+// Hands out the CTA's row pieces one after the other.  The only state is a count of what has been
+// handed out; everything else is recomputed from the launch parameters (registers are scarce here).
 struct Walker {
-  int64_t t, t1, row_i;
-  bool first;
-  __device__ explicit Walker(const RowsParams &p) {
-    first = true;
-    row_i = blockIdx.x;
-    t = first_tile_of(p, blockIdx.x);
-    t1 = first_tile_of(p, (int64_t)blockIdx.x + 1);
+  int rel;  // tiles of the CTA's run handed out so far (interleaved: rows handed out)
+  __device__ Walker() : rel(0) {}
+  __device__ static int64_t run_length(const RowsParams &p) { return p.tiles_q + ((int64_t)blockIdx.x < p.tiles_r ? 1 : 0); }
+  // Row of the first piece, -1 when the CTA has nothing to do.
+  __device__ static int64_t first_row(const RowsParams &p) {
+    if (p.interleaved) return (int64_t)blockIdx.x < p.rows ? (int64_t)blockIdx.x : -1;
+    return run_length(p) > 0 ? quot(p, first_tile_of(p, blockIdx.x), p.tiles_per_row) : -1;
+  }
+  // Row of the piece after `cur` (the piece handed out last), -1 when there is none.
+  __device__ int64_t row_after(const RowsParams &p, const Seg &cur) const {
+    if (p.interleaved) return cur.row + gridDim.x < p.rows ? cur.row + gridDim.x : -1;
+    return rel < run_length(p) ? cur.row + 1 : -1;
   }
   __device__ bool next(const RowsParams &p, Seg &s) {
     if (p.interleaved) {
-      if (row_i >= p.rows) return false;
-      s.row = row_i; s.e_lo = 0; s.e_hi = (int)p.V; s.whole = true; s.starts = true; s.first = first; s.k0 = s.k1 = 0;
-      row_i += gridDim.x;
-      first = false;
+      const int64_t row = (int64_t)blockIdx.x + (int64_t)rel * gridDim.x;
+      if (row >= p.rows) return false;
+      s.row = row; s.e_lo = 0; s.e_hi = (int)p.V; s.whole = true; s.starts = true; s.first = rel == 0; s.k0 = s.k1 = 0;
+      ++rel;
       return true;
     }
-    if (t >= t1) return false;
+    const int64_t len = run_length(p);
+    if (rel >= len) return false;
+    const int64_t t = first_tile_of(p, blockIdx.x) + rel;
     const int64_t row = quot(p, t, p.tiles_per_row), tin = t - row * p.tiles_per_row;
-    const int64_t n = p.tiles_per_row - tin < t1 - t ? p.tiles_per_row - tin : t1 - t;
+    const int64_t n = p.tiles_per_row - tin < len - rel ? p.tiles_per_row - tin : len - rel;
     const int64_t lo = tin * kTile, hi = (tin + n) * kTile;
     s.row = row;
     s.e_lo = (int)(lo < p.V ? lo : p.V);
     s.e_hi = (int)(hi < p.V ? hi : p.V);
     s.starts = tin == 0;
     s.whole = tin == 0 && n == p.tiles_per_row;
-    s.first = first;
+    s.first = rel == 0;
     s.k0 = s.k1 = 0;
     if (!s.whole) {
       s.k0 = cta_of_tile(p, row * p.tiles_per_row);
       s.k1 = cta_of_tile(p, (row + 1) * p.tiles_per_row - 1);
     }
-    first = false;
-    t += n;
+    rel += (int)n;
     return true;
   }
 };
@@ -1016,27 +1050,23 @@ struct Walker {
 // it only needs the mask, and must not wait for anything before its first copy.
 struct SegIter {
   Walker wk;
-  Seg s_next;
   float tau_next;
   bool masked_next;
-  bool has;
   bool with_tau;
-  __device__ SegIter(const RowsParams &p, bool with_tau_) : wk(p), with_tau(with_tau_) { advance(p); }
-  __device__ void advance(const RowsParams &p) {
-    has = wk.next(p, s_next);
+  __device__ SegIter(const RowsParams &p, bool with_tau_) : with_tau(with_tau_) { prefetch(p, Walker::first_row(p)); }
+  __device__ void prefetch(const RowsParams &p, int64_t row) {
     tau_next = p.temp_scalar;
     masked_next = false;
-    if (has) {
-      if (with_tau && p.temps) tau_next = __ldg(p.temps + s_next.row);
-      masked_next = p.mode != kModeSample && p.mask && __ldg(p.mask + s_next.row) == 0;
+    if (row >= 0) {
+      if (with_tau && p.temps) tau_next = __ldg(p.temps + row);
+      masked_next = p.mode != kModeSample && p.mask && __ldg(p.mask + row) == 0;
     }
   }
   __device__ bool next(const RowsParams &p, Seg &s, RowInfo &r) {
-    if (!has) return false;
-    s = s_next;
+    if (!wk.next(p, s)) return false;
     r.tau = tau_next;
     r.masked = masked_next;
-    advance(p);
+    prefetch(p, wk.row_after(p, s));
     r.greedy = p.mode == kModeSample && r.tau == 0.f;
     r.invalid = !r.masked && !r.greedy && !(r.tau > 0.f && r.tau < CUDART_INF_F);
     r.c = r.greedy || r.masked || r.invalid ? 0.f : __fdiv_rn(kLog2e, r.tau);
@@ -1421,59 +1451,73 @@ __global__ void __launch_bounds__(kThreads, 2) rows_kernel(const __grid_constant
               SlowIO io;
               io.acc = acc; io.best = best; io.err = err; io.zsum = 0.f;
               E3_MAKE_CTX(ex);
-              slow_groups<DT, SAMPLER, SAMPLER == 1>(io, ex, owner == tid ? fast_end : s.e_hi, s.e_hi, ri.c, sm);
+              slow_groups<DT, SAMPLER, true>(io, ex, owner == tid ? fast_end : s.e_hi, s.e_hi, ri.c, sm);
               acc = io.acc; best = io.best; err = io.err;
               zextra = io.zsum;
               if (SAMPLER == 0) ethr = gate_threshold(best.enc, acc.nRc);
             }
           }
-          // ---- the streaming form
-          uint4 raw[4];
-          {
-            const uint4 *pv = reinterpret_cast<const uint4 *>(lane_data);
-#pragma unroll
-            for (int i = 0; i < 4; ++i) raw[i] = pv[i ^ rot];
-          }
-          // raw[kVG*gi ...] is group gi ^ ga of the thread (vocabulary order)
+          // ---- the streaming form: one group of 16 entries per turn (a single copy of the code, so that
+          // the loop stays in the instruction cache).  Turn gi works on group gi ^ ga of the thread's 64
+          // bytes and reads its vectors in the order i ^ rot, which keeps the lanes of a quarter warp on
+          // distinct banks.  All lanes of the warp share one reference logit.
           const int ga = kG == 2 ? (rot >> 1) : 0;
-          const Acc saved = acc;
-          const f2 c2 = pack2f(ri.c, ri.c), nRc2 = pack2f(acc.nRc, acc.nRc);
-          float Zg[kG];
-          bool have[kG];
-          bool bad = false;
-#pragma unroll
+          float zl = zextra;  // sampler 1: this thread's share of its block
+#pragma unroll 1
           for (int gi = 0; gi < kG; ++gi) {
-            const int g0 = e_lane + ((gi ^ ga) << 4);
-            have[gi] = g0 + kGroup <= lim;
-            Zg[gi] = 0.f;
-            if (have[gi]) {
-              f2 Zg2;
-              Zg[gi] = hot_group<DT>(&raw[kVG * gi], c2, nRc2, acc.Wa2, acc.Wb2, Zg2);
-              acc.Z2 = add2(acc.Z2, Zg2);
-              bad |= !(Zg[gi] <= kGroupSumMax);
+            const int gn = gi ^ ga;
+            const int g0 = e_lane + (gn << 4);
+            const bool have = g0 + kGroup <= lim;
+            uint4 raw[kVG];
+            {
+              const uint4 *pv = reinterpret_cast<const uint4 *>(lane_data) + gn * kVG;
+#pragma unroll
+              for (int i = 0; i < kVG; ++i) raw[i] = pv[(i ^ rot) & (kVG - 1)];
             }
-          }
-          if (SAMPLER == 1) bad = __any_sync(0xffffffffu, bad);
-          if (bad) {
-            StepIO io;
-            io.acc = saved; io.err = err; io.Zextra = zextra;
-            io.Zg[0] = 0.f; io.Zg[kG - 1] = 0.f;
-            int hv = 0;
-#pragma unroll
-            for (int gi = 0; gi < kG; ++gi) hv |= (have[gi] ? 1 : 0) << (gi ^ ga);
-            redo_step<DT, SAMPLER == 1>(io, lane_data, hv, ri.c);
-            acc = io.acc; err = io.err; zextra = io.Zextra;
-#pragma unroll
-            for (int gi = 0; gi < kG; ++gi) Zg[gi] = io.Zg[gi ^ ga];
-            if (SAMPLER == 0) ethr = gate_threshold(best.enc, acc.nRc);
-          }
-          if (SAMPLER == 0) {
-#pragma unroll
-            for (int gi = 0; gi < kG; ++gi) {
-              const int g0 = e_lane + ((gi ^ ga) << 4);
+            float Zg = 0.f;
+            f2 Zg2 = pack2f(0.f, 0.f);
+            f2 Wa_in = acc.Wa2, Wb_in = acc.Wb2;
+#pragma unroll 1
+            for (int attempt = 0;; ++attempt) {
+              if (have) Zg = hot_group<DT>(raw, pack2f(ri.c, ri.c), pack2f(acc.nRc, acc.nRc), acc.Wa2, acc.Wb2, Zg2);
+              if (!__any_sync(0xffffffffu, have && !(Zg <= kGroupSumMax))) break;
+              // the reference is stale for some lane (or a value is not finite)
+              acc.Wa2 = Wa_in; acc.Wb2 = Wb_in;
+              const float gm = have ? group_max<DT>(raw) : -CUDART_INF_F;
+              const float newR = dec_float(__reduce_max_sync(0xffffffffu, enc_float(gm)));
+              const float nRc = -newR * ri.c;
+              if (attempt == 0 && newR > acc.R && newR < CUDART_INF_F && fabsf(nRc) < CUDART_INF_F) {
+                // move the warp's reference up to the largest logit of this turn and repeat the group
+                const float d = nRc - acc.nRc;
+                const float f = acc.R == -CUDART_INF_F ? 0.f : ex2f(d);
+                const f2 ff = pack2f(f, f);
+                acc.Wa2 = mul2(ff, fma2(pack2f(d, d), acc.Z2, acc.Wa2));
+                acc.Wb2 = mul2(ff, acc.Wb2);
+                acc.Z2 = mul2(ff, acc.Z2);
+                if (f == 0.f) acc.Z2 = acc.Wa2 = acc.Wb2 = pack2f(0.f, 0.f);
+                acc.R = newR; acc.nRc = nRc;
+                zl *= f;
+                Wa_in = acc.Wa2; Wb_in = acc.Wb2;
+                if (SAMPLER == 0) ethr = gate_threshold(best.enc, acc.nRc);
+                continue;
+              }
+              // NaN, +inf or numbers outside the fp32 range: the careful form sorts it out
+              StepIO io;
+              io.acc = acc; io.err = err; io.Zextra = zl;
+              io.Zg[0] = 0.f; io.Zg[kG - 1] = 0.f;
+              redo_step<DT, true>(io, lane_data, have ? (1 << gn) : 0, ri.c);
+              acc = io.acc; err = io.err; zl = io.Zextra;
+              Zg = io.Zg[gn];
+              Zg2 = pack2f(0.f, 0.f);  // the careful form has added the group already
+              if (SAMPLER == 0) ethr = gate_threshold(best.enc, acc.nRc);
+              break;
+            }
+            acc.Z2 = add2(acc.Z2, Zg2);
+            zl += Zg;
+            if (SAMPLER == 0) {
               const uint4 cb = philox(rk, (uint32_t)g0 >> 4, grow, p.ctr_lo, p.ctr_hi8 | 0u);
-              const bool over = Zg[gi] > ethr;
-              const bool flag = have[gi] && (any_ff4(cb) != 0u || over);
+              const bool over = Zg > ethr;
+              const bool flag = have && (any_ff4(cb) != 0u || over);
               const uint32_t ballot = __ballot_sync(0xffffffffu, flag);
               if (ballot != 0u) {
                 if (flag) {
@@ -1482,7 +1526,7 @@ __global__ void __launch_bounds__(kThreads, 2) rows_kernel(const __grid_constant
                   uint4 *ent = reinterpret_cast<uint4 *>(queue + kQueueHdrBytes + pos * F::kEntryBytes);
                   ent[0] = cb;
 #pragma unroll
-                  for (int i = 0; i < kVG; ++i) ent[1 + ((i ^ rot) & (kVG - 1))] = raw[kVG * gi + i];
+                  for (int i = 0; i < kVG; ++i) ent[1 + ((i ^ rot) & (kVG - 1))] = raw[i];
                 }
                 qn += __popc(ballot);
                 if (qn >= kDrainAt) {
@@ -1497,12 +1541,7 @@ __global__ void __launch_bounds__(kThreads, 2) rows_kernel(const __grid_constant
               }
             }
           }
-          if (SAMPLER == 1) {
-            float zl = zextra;
-#pragma unroll
-            for (int gi = 0; gi < kG; ++gi) zl += Zg[gi];
-            block_step<DT>(zl, e_lane >> 8, acc.nRc, rk, grow, p.ctr_lo, p.ctr_hi8, bs, lane);
-          }
+          if (SAMPLER == 1) block_step<DT>(zl, e_lane >> 8, acc.nRc, rk, grow, p.ctr_lo, p.ctr_hi8, bs, lane);
         } else if (ri.greedy) {
           SlowIO io;
           io.acc = acc; io.best = best; io.err = err; io.zsum = 0.f;
@@ -1514,7 +1553,7 @@ __global__ void __launch_bounds__(kThreads, 2) rows_kernel(const __grid_constant
           SlowIO io;
           io.acc = acc; io.best = best; io.err = err; io.zsum = 0.f;
           E3_MAKE_CTX(ex);
-          slow_groups<DT, SAMPLER, SAMPLER == 1>(io, ex, e_lane < s.e_hi ? e_lane : s.e_hi, s.e_hi, ri.c, sm);
+          slow_groups<DT, SAMPLER, true>(io, ex, e_lane < s.e_hi ? e_lane : s.e_hi, s.e_hi, ri.c, sm);
           acc = io.acc; best = io.best; err = io.err;
           if (SAMPLER == 1) block_step<DT>(io.zsum, e_lane >> 8, acc.nRc, rk, grow, p.ctr_lo, p.ctr_hi8, bs, lane);
         }
@@ -1772,6 +1811,7 @@ cudaError_t launch_one(RowsParams p, void *workspace, size_t workspace_bytes, cu
   p.tiles_per_row = (p.V + kTile - 1) / kTile;
   const int64_t tiles = p.rows * p.tiles_per_row;
   p.narrow = tiles < (int64_t(1) << 31) ? 1 : 0;
+  if (tiles / slots >= (int64_t(1) << 30)) return cudaErrorInvalidValue;  // per-CTA tile counts are kept in 32 bits
   const bool can_cut = workspace != nullptr && workspace_bytes >= rows_workspace_bytes();
   // With a response mask the cost of a row is not known on the host: spread whole rows round-robin.
   p.interleaved = (!can_cut || (p.mask != nullptr && p.rows >= 4 * slots)) ? 1 : 0;
