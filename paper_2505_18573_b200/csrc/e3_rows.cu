@@ -1359,6 +1359,12 @@ __global__ void __launch_bounds__(kThreads, 2) rows_kernel(const __grid_constant
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
+  // Programmatic dependent launch: this grid may have been started while the kernel before it in the
+  // stream was still finishing (launch latency, block start-up and the set-up above then overlap with that
+  // kernel's tail).  Nothing in global memory may be touched before the wait below, which returns once the
+  // earlier kernel has completed and its writes are visible; the grid behind this one may start likewise.
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
   const int full_end = (int)(p.V & ~(int64_t)15);  // entries covered by full groups
 
@@ -1820,8 +1826,17 @@ cudaError_t launch_one(RowsParams p, void *workspace, size_t workspace_bytes, cu
   p.tiles_r = tiles % grid;
   p.ws_pieces = can_cut ? static_cast<unsigned char *>(workspace) : nullptr;
   p.call_id = next_call_id();
-  rows_kernel<DT, SAMPLER, RING><<<(unsigned)grid, kThreads, dyn_smem_bytes<DT, SAMPLER, RING>(), stream>>>(p);
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)grid);
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = dyn_smem_bytes<DT, SAMPLER, RING>();
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, rows_kernel<DT, SAMPLER, RING>, p);
 }
 
 }  // namespace
