@@ -45,6 +45,9 @@ ROWS, V, DECODE_STEPS, RING = 512, 151936, 256, 8
 GROUP = 8
 METRIC = "logit rows/s, fused sample+entropy, V=151,936"
 UNIT = "rows/s"
+# dram__bytes_read.sum + dram__bytes_write.sum of one e3_sample launch of this workload (ncu capture summarised in
+# profiles/rows_kernel_c2_ncu_full.txt); only for the kernel variant that was captured.
+NCU_TRAFFIC_BYTES = {1: 165.8e6}
 WORKLOAD = "rollout decode step: 512 rows (64 prompts x 8 rollouts) x V=151,936 bf16, 256 decode steps"
 
 
@@ -381,7 +384,8 @@ def main():
             "roofline": {"bound": "hbm", "kernel": f"rows_kernel (e3_sample, sampler {args.sampler}, bf16)",
                          "achieved": achieved, "peak": peak,
                          "peak_kind": peak_kind, "unit": "GB/s", "frac": achieved / peak, "frac_of_8TBs": achieved / 8000.0,
-                         "us_per_launch": launch_s * 1e6, "bytes_per_launch": bytes_per_launch, "traffic": None},
+                         "us_per_launch": launch_s * 1e6, "bytes_per_launch": bytes_per_launch,
+                         "traffic": NCU_TRAFFIC_BYTES.get(args.sampler)},
             "training_side": {"ms_per_step": ms_tail / args.steps, "unmasked_rows": unmasked,
                               "GBps_incl_small_kernels_and_sync": train_bytes / (ms_tail * 1e-3 / args.steps) / 1e9},
             "kernels": {k: {"us_per_launch": v, "GBps": bytes_per_launch / v / 1e3, "frac": bytes_per_launch / v / 1e3 / peak}
