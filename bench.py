@@ -175,7 +175,7 @@ def run_reference(args, rank: int):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=30)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--sampler", type=int, default=1, choices=[0, 1],
                     help="0 = one Gumbel per vocabulary entry, 1 = one Gumbel per block of 256 entries (default)")

@@ -1015,7 +1015,8 @@ struct Walker {
     if (p.interleaved) return cur.row + gridDim.x < p.rows ? cur.row + gridDim.x : -1;
     return rel < run_length(p) ? cur.row + 1 : -1;
   }
-  __device__ bool next(const RowsParams &p, Seg &s) {
+  // with_range: also work out which CTAs hold the row's first and last tile (only the finishing warp asks)
+  __device__ bool next(const RowsParams &p, Seg &s, bool with_range) {
     if (p.interleaved) {
       const int64_t row = (int64_t)blockIdx.x + (int64_t)rel * gridDim.x;
       if (row >= p.rows) return false;
@@ -1036,7 +1037,7 @@ struct Walker {
     s.whole = tin == 0 && n == p.tiles_per_row;
     s.first = rel == 0;
     s.k0 = s.k1 = 0;
-    if (!s.whole) {
+    if (!s.whole && with_range) {
       s.k0 = cta_of_tile(p, row * p.tiles_per_row);
       s.k1 = cta_of_tile(p, (row + 1) * p.tiles_per_row - 1);
     }
@@ -1052,8 +1053,11 @@ struct SegIter {
   Walker wk;
   float tau_next;
   bool masked_next;
-  bool with_tau;
-  __device__ SegIter(const RowsParams &p, bool with_tau_) : with_tau(with_tau_) { prefetch(p, Walker::first_row(p)); }
+  bool with_tau, with_range;
+  __device__ SegIter(const RowsParams &p, bool with_tau_, bool with_range_ = false)
+      : with_tau(with_tau_), with_range(with_range_) {
+    prefetch(p, Walker::first_row(p));
+  }
   __device__ void prefetch(const RowsParams &p, int64_t row) {
     tau_next = p.temp_scalar;
     masked_next = false;
@@ -1063,7 +1067,7 @@ struct SegIter {
     }
   }
   __device__ bool next(const RowsParams &p, Seg &s, RowInfo &r) {
-    if (!wk.next(p, s)) return false;
+    if (!wk.next(p, s, with_range)) return false;
     r.tau = tau_next;
     r.masked = masked_next;
     prefetch(p, wk.row_after(p, s));
@@ -1659,7 +1663,7 @@ __global__ void __launch_bounds__(kThreads, 2) rows_kernel(const __grid_constant
     }
   } else {
     // ------------------------------------------------------------------ finishing warp
-    SegIter it(p, true);
+    SegIter it(p, true, true);
     Seg s;
     RowInfo ri;
     uint32_t n = 0;
