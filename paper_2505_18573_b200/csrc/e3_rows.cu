@@ -6,36 +6,43 @@
 // persistent grid (two per SM) takes an equal, contiguous run of tiles, so all CTAs stream the
 // same number of bytes whatever the number of rows.  A run covers the tail of one row, some
 // whole rows and the head of another.  Whole rows are finished by the CTA itself.  For a row
-// that is cut, every CTA holding a piece stores its partial state in the caller's workspace and
-// announces it with a compare-and-swap on a per-row arrival word tagged with a per-call id; the
-// CTA whose announcement completes the row merges the pieces and writes the outputs.  Nobody
-// waits for anybody.  (With a response mask, and when no workspace is given, CTAs take whole
-// rows round-robin instead.)
+// that is cut, every CTA holding a piece stores its partial state in the caller's workspace (64-bit
+// words tagged with a per-call id), issues a sequentially consistent fence and then looks for the
+// row's other pieces: the CTA whose fence comes last finds them all, merges them and writes the
+// outputs.  Nobody waits for anybody.  (With a response mask, and when no workspace is given, CTAs
+// take whole rows round-robin instead.)
 //
 // Inside a CTA: one thread issues bulk asynchronous copies (cp.async.bulk, no multicast) of 16 KiB
 // into a 4-stage shared-memory ring guarded by mbarriers; eight warps consume the ring, each
 // thread 64 contiguous bytes per stage (read in a swizzled vector order that is free of bank
 // conflicts); one warp finishes rows (merges the eight warp states, fp64 epilogue, piece protocol)
-// so that the consumers never stall on it.  Every role looks one row ahead for its temperature and
-// mask.  Every mbarrier wait is bounded: when a wait runs out the CTA stops waiting altogether,
-// finishes its fixed sequence of steps on whatever data it has and marks its rows invalid.
+// so that the consumers never stall on it.  Consumers and the finishing warp look one row ahead for
+// the temperature; the copy-issuing thread never needs it.  Every mbarrier wait is bounded: when a
+// wait runs out the CTA stops waiting altogether, finishes its fixed sequence of steps on whatever
+// data it has and marks its rows invalid.  The kernel is launched with programmatic stream
+// serialization: its set-up overlaps the tail of the kernel before it in the stream, and it touches
+// global memory only after griddepcontrol.wait.
 //
-// Numerics.  Each thread keeps a reference logit R and the sums Z = sum 2^t, W = sum 2^t * t with
-// t = z*c - R*c and c = log2(e)/tau, two entries per instruction (packed fp32).  The streaming loop
-// never looks for the maximum: R is taken from the first entries of the row piece and stays until a
-// group sum leaves the safe range, which sends that group through a careful out-of-line form that
-// moves R (and also deals with NaN and infinities).  -inf logits are clamped to a huge negative finite
-// value on the way in, which gives them weight 0 without special cases.  States merge
-// associatively; the per-row result is formed in fp64:
+// Numerics.  All lanes of a warp share a reference logit R; each thread keeps the sums Z = sum 2^t,
+// W = sum 2^t * t with t = z*c - R*c and c = log2(e)/tau, two entries per instruction (packed fp32).
+// The streaming loop never looks for the maximum: R is taken from the first entries of the row piece;
+// when the sum of a group of 16 leaves the safe range (some t above 1..5) the warp moves R up to the
+// largest logit of the current turn, rescales its sums and repeats the group.  R therefore stays
+// close to the largest logit seen, which keeps W/Z small and the entropy free of cancellation.
+// -inf logits are clamped to a huge negative finite value on the way in, which gives them weight 0
+// without special cases; NaN and +inf end up in a careful out-of-line form that flags the row.
+// States merge associatively; the per-row result is formed in fp64:
 // H = ln Z - ln2 * W / Z,  ln p_tok = (z_tok*c - M) ln2 - ln Z.
 //
 // Sampler 0 (one Gumbel per vocabulary entry).  u_i has 8 coarse + 32 fine bits.  An entry can
 // only win if its coarse byte is 255 (g_i >= 5.5432) or if z_i/tau exceeds the best score so
 // far minus 5.5432; the second condition is tested on the group sum of 2^t, which bounds every
 // term from above.  Groups that pass are copied (coarse bytes and logits) into a per-warp queue
-// in shared memory with ballot-compacted positions; when 32 are waiting the warp evaluates them,
-// one per lane: an fp32 upper bound first, the survivors in fp64 with the same expression order
-// as the definition.  The token never depends on the gating.
+// in shared memory with ballot-compacted positions; when 32 are waiting the warp scores them, one
+// per lane, in fp32 with a proven error bound, and every thread keeps its three leaders.  The
+// finishing warp takes the fp32 leader when it is ahead by more than two error bounds; otherwise
+// it evaluates the contenders in fp64 with the expression order of the definition (or looks at the
+// whole row again when there are three or more).  The token never depends on the gating or on fp32.
 //
 // Sampler 1 (one Gumbel per block of 256 entries).  8 (bf16) or 16 (fp32) neighbouring lanes hold
 // one block per step; their sums are added with shuffles, each lane parks one block and all lanes

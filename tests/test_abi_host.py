@@ -48,7 +48,7 @@ def test_device_calls_reject_bad_arguments_on_the_host(e3):
     assert L.e3_sample(None, 0, 1, 1 << 31, 1 << 31, None, 0, 0, 0, 0, None, None, None, None, 0, None) == 1
     assert L.e3_sample(None, 0, 0, 8, 8, None, 0, 0, 0, 0, None, None, None, None, 0, None) == 0   # rows == 0
     assert L.e3_sample(None, 0, 0, 8, 8, None, 0, 1 << 56, 0, 0, None, None, None, None, 0, None) == 1
-    assert L.e3_sample(None, 0, 0, 8, 8, None, 0, 0, 0, 2, None, None, None, None, 0, None) == 1   # sampler
+    assert L.e3_sample(None, 0, 0, 8, 8, None, 0, 0, 0, 3, None, None, None, None, 0, None) == 1   # sampler
     assert L.e3_sample(1024, 0, 1, 8, 8, None, 0, 0, 0, 0, None, None, None, None, 0, None) == 1   # temps NULL
     assert L.e3_sample(1026, 0, 1, 8, 8, 1024, 0, 0, 0, 0, 1024, None, None, None, 0, None) == 3   # misaligned
     assert L.e3_token_logp_entropy(None, 0, 0, 8, 8, None, None, None, 1.0, None, None, None, 0, None) == 0
