@@ -144,6 +144,24 @@ def token_logp_entropy(logits: np.ndarray, targets: np.ndarray, mask=None, temps
     return tuple(outs)
 
 
+def token_logp_entropy_backward(logits: np.ndarray, targets: np.ndarray, g_logp=None, g_ent=None, mask=None, temps=None,
+                                temp_scalar: float = 1.0) -> np.ndarray:
+    """Gradient with respect to the logits, float64 [rows, V]."""
+    ptr, dt, rows, V, stride = _logits_args(logits)
+    targets = np.ascontiguousarray(targets, dtype=np.int32)
+    mask = None if mask is None else np.ascontiguousarray(mask, dtype=np.uint8)
+    temps = None if temps is None else np.ascontiguousarray(temps, dtype=np.float32)
+    g_logp = None if g_logp is None else np.ascontiguousarray(g_logp, dtype=np.float32)
+    g_ent = None if g_ent is None else np.ascontiguousarray(g_ent, dtype=np.float32)
+    out = np.empty((rows, V), np.float64)
+    rc = lib().e3o_token_logp_entropy_backward(ptr, dt, C.c_int64(rows), C.c_int64(V), C.c_int64(stride), _p(targets),
+                                               _p(mask), _p(temps), C.c_float(temp_scalar), _p(g_logp), _p(g_ent),
+                                               _p(out))
+    if rc != 0:
+        raise ValueError("e3o_token_logp_entropy_backward: invalid argument")
+    return out
+
+
 def masked_mean_entropy(ent: np.ndarray, mask=None):
     """Returns (mean, count) as Python floats."""
     ent = np.ascontiguousarray(ent, dtype=np.float32)

@@ -26,6 +26,8 @@
  *   Sec. 2 / Sec. 5.1 (tokens are drawn from softmax(z/tau))   -> e3o_sample
  *   Sec. 4.2 ("logits are also divided by the temperature
  *             during forward propagation after sampling")     -> e3o_token_logp_entropy
+ *   Sec. 3.1 objective, Sec. 4.2 entropy regulariser (chain rule
+ *             through the softmax of App. A)                   -> e3o_token_logp_entropy_backward
  *   Sec. 4.2 (H_init, H_t: average entropy of a batch)         -> e3o_masked_mean_entropy
  *   Eq. "adv" (Sec. 3.1)                                       -> e3o_group_advantage
  *   Algorithm 1 (Sec. 4.1)                                     -> e3o_allocate_budget
@@ -350,6 +352,59 @@ int e3o_token_logp_entropy(const void *logits, int dt, int64_t rows, int64_t V, 
       if (out_logp) out_logp[r] = lp;
       if (out_ent) out_ent[r] = en;
       if (out_ent_dec) out_ent_dec[r] = ed;
+    }
+    free(s);
+  }
+  return 0;
+}
+
+/* ------------------------------------------------------------------------- */
+/* Gradient of the training-side outputs with respect to the logits.  The     */
+/* objective of Sec. 3.1 depends on the logits through ln pi(o_t), the        */
+/* entropy-regularised objective discussed in Sec. 4.2 also through H; with   */
+/* p = softmax(z / tau), beta = 1/tau (App. A) the chain rule through the     */
+/* softmax gives                                                              */
+/*   d ln p_tok / d z_i = beta (1[i == tok] - p_i)                            */
+/*   d H        / d z_i = -beta p_i (ln p_i + H)                              */
+/* so that, for upstream gradients g_logp and g_ent of a row,                 */
+/*   dlogits_i = beta [ g_logp (1[i == tok] - p_i) - g_ent p_i (ln p_i + H) ].*/
+/* Rows with mask == 0 get zeros; an invalid row or a target outside [0, V)   */
+/* gives NaN.  Entries with p_i = 0 (logit -inf) get 0 from the entropy term. */
+/* Pins: central differences of e3o_token_logp_entropy itself; the gradient   */
+/* sums to zero over a row; an autograd library on tiny rows.                 */
+/* ------------------------------------------------------------------------- */
+int e3o_token_logp_entropy_backward(const void *logits, int dt, int64_t rows, int64_t V, int64_t row_stride,
+                                    const int32_t *targets, const uint8_t *mask, const float *temps,
+                                    float temp_scalar, const float *g_logp, const float *g_ent,
+                                    double *out_dlogits /* [rows, V] dense */) {
+  if (rows < 0 || V < 1 || row_stride < V || (dt != E3O_F32 && dt != E3O_BF16)) return 1;
+  size_t esz = dt == E3O_F32 ? 4 : 2;
+#pragma omp parallel
+  {
+    double *s = (double *)malloc(sizeof(double) * (size_t)V);
+#pragma omp for schedule(dynamic, 1)
+    for (int64_t r = 0; r < rows; ++r) {
+      double *d = out_dlogits + (size_t)r * (size_t)V;
+      if (mask && !mask[r]) {
+        for (int64_t i = 0; i < V; ++i) d[i] = 0.0;
+        continue;
+      }
+      const char *row = (const char *)logits + (size_t)r * (size_t)row_stride * esz;
+      double tau = temps ? (double)temps[r] : (double)temp_scalar;
+      row_stats st;
+      int32_t t = targets[r];
+      if (row_softmax_stats(row, dt, V, tau, s, &st) != 0 || t < 0 || t >= V) {
+        for (int64_t i = 0; i < V; ++i) d[i] = NAN;
+        continue;
+      }
+      double beta = 1.0 / tau, H = st.H_def, lnZ = log(st.Z);
+      double gl = g_logp ? (double)g_logp[r] : 0.0, ge = g_ent ? (double)g_ent[r] : 0.0;
+      for (int64_t i = 0; i < V; ++i) {
+        double lnp = s[i] - st.m - lnZ;
+        double p = exp(lnp);
+        double ent_term = p > 0.0 ? p * (lnp + H) : 0.0;
+        d[i] = beta * (gl * ((i == t ? 1.0 : 0.0) - p) - ge * ent_term);
+      }
     }
     free(s);
   }

@@ -542,3 +542,56 @@ def test_annealing_schedule_end_points():
     s = oracle.make_sched(tau=1.0, H_init=H0, t=t_max, t_anneal=t_a, t_max=t_max, eta=eta, V=151936)
     denom = math.log(151936) + math.log(math.log(151936))
     assert oracle.update_temperature(s, H0) == pytest.approx(1 + math.log(eta) / denom, rel=1e-13)
+
+
+# ----------------------------------------------------------------------------------------------
+# gradient of log-probability and entropy with respect to the logits
+# ----------------------------------------------------------------------------------------------
+def test_backward_matches_central_differences_of_the_forward_oracle(oracle_mod):
+    o = oracle_mod
+    rng = np.random.default_rng(5)
+    rows, V = 3, 9
+    z = rng.normal(size=(rows, V)).astype(np.float32) * 2
+    z[1, 4] = -np.inf                                   # an entry without mass
+    targets = np.array([2, 0, 8], np.int32)
+    temps = np.array([0.7, 1.0, 1.9], np.float32)
+    g_lp = np.array([1.0, -0.5, 2.0], np.float32)
+    g_en = np.array([0.25, 1.0, -3.0], np.float32)
+    d = o.token_logp_entropy_backward(z, targets, g_lp, g_en, temps=temps)
+    h = 2.0 ** -7                                       # exactly representable step, fp32 logits stay exact
+    for r in range(rows):
+        for i in range(V):
+            if not np.isfinite(z[r, i]):
+                assert d[r, i] == 0.0
+                continue
+            zp, zm = z.copy(), z.copy()
+            zp[r, i] += h; zm[r, i] -= h
+            lp_p, en_p, _ = o.token_logp_entropy(zp, targets, temps=temps)
+            lp_m, en_m, _ = o.token_logp_entropy(zm, targets, temps=temps)
+            num = (g_lp[r] * (lp_p[r] - lp_m[r]) + g_en[r] * (en_p[r] - en_m[r])) / (2 * h)
+            assert d[r, i] == pytest.approx(num, abs=2e-4), (r, i)   # O(h^2) truncation
+
+
+def test_backward_sums_to_zero_and_matches_autograd(oracle_mod):
+    import torch
+    o = oracle_mod
+    rng = np.random.default_rng(6)
+    rows, V = 4, 50
+    z = rng.normal(size=(rows, V)).astype(np.float32) * 3
+    targets = rng.integers(0, V, size=rows).astype(np.int32)
+    g_lp = rng.normal(size=rows).astype(np.float32)
+    g_en = rng.normal(size=rows).astype(np.float32)
+    mask = np.array([1, 0, 1, 1], np.uint8)
+    d = o.token_logp_entropy_backward(z, targets, g_lp, g_en, mask=mask, temp_scalar=1.3)
+    assert np.all(d[1] == 0.0)
+    assert np.abs(d.sum(axis=1)).max() < 1e-12          # both terms are orthogonal to the all-ones direction
+    zt = torch.tensor(z, dtype=torch.float64, requires_grad=True)
+    logp_all = torch.log_softmax(zt / float(np.float32(1.3)), dim=1)
+    lp = logp_all[torch.arange(rows), torch.tensor(targets, dtype=torch.long)]
+    H = -(logp_all.exp() * logp_all).sum(dim=1)
+    m = torch.tensor(mask, dtype=torch.float64)
+    (m * (torch.tensor(g_lp, dtype=torch.float64) * lp + torch.tensor(g_en, dtype=torch.float64) * H)).sum().backward()
+    assert np.abs(d - zt.grad.numpy()).max() < 1e-12
+    # out-of-range target and invalid temperature
+    bad = o.token_logp_entropy_backward(z[:1], np.array([V], np.int32), g_lp[:1], g_en[:1])
+    assert np.isnan(bad).all()
