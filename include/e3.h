@@ -132,6 +132,30 @@ E3_API e3_status e3_token_logp_entropy(const void *logits, e3_dtype dt, int64_t 
                                 void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * Backward of e3_token_logp_entropy.  The objective of Sec. 3.1 depends on the logits through
+ * ln pi(o_t), and the entropy-regularised objective discussed in Sec. 4.2 also through the entropy H;
+ * with p = softmax(logits[r] / tau_r), beta = 1/tau_r (App. A) the chain rule through the softmax gives,
+ * for every row with mask[r] != 0,
+ *   dlogits[r, i] = beta ( g_logp[r] (1[i == targets[r]] - p_i)  -  g_ent[r] p_i (ln p_i + H_r) ).
+ * Rows with mask[r] == 0 get zeros.  A row whose temperature, target or forward outputs are not usable
+ * (tau <= 0 or not finite, target outside [0, V), logp or ent NaN) gets NaN.
+ *
+ *   logits, dt, rows, V, row_stride, targets, mask, temps, temp_scalar   as in the forward call
+ *   logp, ent     device float [rows]: the forward call's outputs for the same arguments (the row's
+ *                 normaliser is taken from them: ln p_i = (z_i - z_tok)/tau + logp)
+ *   g_logp, g_ent device float [rows]: upstream gradients; NULL = all zero
+ *   dlogits       device, same element type as logits, row r starts at element r * dlogits_stride
+ *                 (dlogits_stride >= V); must not overlap logits.  Rows and strides that are 16-byte
+ *                 aligned on both sides take the vectorised path.
+ * No workspace.  One pass: V entries read and V written per row.
+ */
+E3_API e3_status e3_token_logp_entropy_backward(const void *logits, e3_dtype dt, int64_t rows, int64_t V,
+                                         int64_t row_stride, const int32_t *targets, const uint8_t *mask,
+                                         const float *temps, float temp_scalar, const float *logp, const float *ent,
+                                         const float *g_logp, const float *g_ent, void *dlogits,
+                                         int64_t dlogits_stride, void *stream);
+
+/*
  * Batch entropy H_t of the scheduler (Sec. 4.2: "average entropy" of a batch), read as the mean
  * over all response tokens: out_mean = sum_j mask[j] ent[j] / sum_j mask[j], accumulated in
  * fp64 in a fixed order.  out_count = sum_j mask[j].  count == 0 gives mean NaN.

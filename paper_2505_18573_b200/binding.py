@@ -22,6 +22,7 @@ E3_CALL_SAMPLE, E3_CALL_TOKEN_LOGP_ENTROPY, E3_CALL_MASKED_MEAN_ENTROPY = 0, 1, 
 E3_SAMPLE_BLOCK = 256
 
 EXPORTS = ("e3_status_string", "e3_workspace_bytes", "e3_sample", "e3_token_logp_entropy",
+           "e3_token_logp_entropy_backward",
            "e3_masked_mean_entropy", "e3_masked_mean_entropy_static", "e3_group_advantage", "e3_allocate_budget", "e3_update_temperature",
            "e3_anneal_target")
 
@@ -61,6 +62,10 @@ def lib() -> C.CDLL:
         L.e3_token_logp_entropy.argtypes = [C.c_void_p, C.c_int, C.c_int64, C.c_int64, C.c_int64, C.c_void_p,
                                             C.c_void_p, C.c_void_p, C.c_float, C.c_void_p, C.c_void_p, C.c_void_p,
                                             C.c_size_t, C.c_void_p]
+        L.e3_token_logp_entropy_backward.restype = C.c_int
+        L.e3_token_logp_entropy_backward.argtypes = [C.c_void_p, C.c_int, C.c_int64, C.c_int64, C.c_int64, C.c_void_p,
+                                                     C.c_void_p, C.c_void_p, C.c_float, C.c_void_p, C.c_void_p,
+                                                     C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p]
         L.e3_masked_mean_entropy.restype = C.c_int
         L.e3_masked_mean_entropy.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p,
                                              C.c_size_t, C.c_void_p]
@@ -189,6 +194,29 @@ def e3_token_logp_entropy(logits, targets, mask=None, temps=None, temp_scalar: f
                                      workspace.numel() * workspace.element_size(), sh)
     _check("e3_token_logp_entropy", st)
     return out_logp, out_ent
+
+
+def e3_token_logp_entropy_backward(logits, targets, logp, ent, g_logp=None, g_ent=None, mask=None, temps=None,
+                                   temp_scalar: float = 1.0, out=None, stream=None):
+    """Gradient of the training-side outputs with respect to the logits: tensor like ``logits``."""
+    dt, rows, V, stride = _logits_desc(logits)
+    for name, t in (("targets", targets), ("logp", logp), ("ent", ent), ("g_logp", g_logp), ("g_ent", g_ent),
+                    ("mask", mask), ("temps", temps)):
+        _dev(t, name)
+        if t is not None and (t.numel() != rows or not t.is_contiguous()):
+            raise ValueError(f"{name} must be contiguous with one entry per row")
+    if targets.dtype != torch.int32 or logp.dtype != torch.float32 or ent.dtype != torch.float32:
+        raise ValueError("targets must be int32, logp and ent float32")
+    if out is None:
+        out = torch.empty((rows, V), dtype=logits.dtype, device=logits.device)
+    _, orows, oV, ostride = _logits_desc(out)
+    if out.dtype != logits.dtype or orows != rows or oV != V:
+        raise ValueError("out must have the shape and dtype of logits")
+    st = lib().e3_token_logp_entropy_backward(_ptr(logits), dt, rows, V, stride, _ptr(targets), _ptr(mask), _ptr(temps),
+                                              float(temp_scalar), _ptr(logp), _ptr(ent), _ptr(g_logp), _ptr(g_ent),
+                                              _ptr(out), ostride, _stream(stream))
+    _check("e3_token_logp_entropy_backward", st)
+    return out
 
 
 def e3_masked_mean_entropy(ent, mask=None, out=None, workspace=None, stream=None):
