@@ -365,6 +365,12 @@ def main():
         "e3_token_logp_entropy": time_alone(lambda d: e3.e3_token_logp_entropy(ring[d % RING], targets1, temps=temps,
                                                                                  out_logp=logp, out_ent=ent)),
     }
+    # backward of the training-side pass over one ring buffer (reads and writes 155.6 MB each)
+    g1 = torch.ones(ROWS, dtype=torch.float32, device=dev)
+    dz = torch.empty((ROWS, V), dtype=torch.bfloat16, device=dev)
+    e3.e3_token_logp_entropy(ring[0], targets1, temps=temps, out_logp=logp, out_ent=ent)
+    bwd_us = time_alone(lambda d: e3.e3_token_logp_entropy_backward(ring[d % RING], targets1, logp, ent, g1, g1,
+                                                                    temps=temps, out=dz))
 
     if rank == 0:
         peak, peak_kind = _peaks()
@@ -390,6 +396,9 @@ def main():
                               "GBps_incl_small_kernels_and_sync": train_bytes / (ms_tail * 1e-3 / args.steps) / 1e9},
             "kernels": {k: {"us_per_launch": v, "GBps": bytes_per_launch / v / 1e3, "frac": bytes_per_launch / v / 1e3 / peak}
                         for k, v in alone.items()},
+            "backward": {"kernel": "e3_token_logp_entropy_backward (next row of the scope table, not part of the step)",
+                         "us_per_launch": bwd_us, "GBps_read_plus_write": 2 * ROWS * V * 2 / bwd_us / 1e3,
+                         "frac": 2 * ROWS * V * 2 / bwd_us / 1e3 / peak},
             "e2e": e2e,
             "gpu_launches": launches_per_step * args.steps,
             "clocks": clocks.summary(),

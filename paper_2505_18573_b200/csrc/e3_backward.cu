@@ -8,6 +8,7 @@
 //
 // Work items are (row, segment of 8,192 entries); a grid of a few CTAs per SM walks them with a stride,
 // each thread moving 16-byte vectors (8 bf16 or 4 fp32 logits) with streaming loads and stores.
+#include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <math_constants.h>
 #include <stdint.h>
@@ -49,11 +50,15 @@ __device__ __forceinline__ float ex2f(float x) {
   return y;
 }
 
-__device__ __forceinline__ float grad_entry(const RowCoef &k, float z, int i) {
-  const float t = fmaf(z - k.zt, k.c, k.lp2);  // log2 p_i
+// Gradient entry without the 1[i == tok] part: -p_i (beta g_logp + beta g_ent (ln p_i + H)).
+// log2 p_i is kept above -16384, so that an entry without weight (-inf logit) gives 0 and not 0 * inf.
+__device__ __forceinline__ float grad_entry_no_target(const RowCoef &k, float z) {
+  const float t = fmaxf(fmaf(z - k.zt, k.c, k.lp2), -16384.f);
   const float p = ex2f(t);
-  const float ent_term = p > 0.f ? p * fmaf(t, kLn2, k.H) : 0.f;  // p (ln p + H); no weight, no term
-  return fmaf(k.a_lp, (i == k.tok ? 1.f : 0.f) - p, -k.a_en * ent_term);
+  return -p * fmaf(k.a_en, fmaf(t, kLn2, k.H), k.a_lp);
+}
+__device__ __forceinline__ float grad_entry(const RowCoef &k, float z, int i) {
+  return grad_entry_no_target(k, z) + (i == k.tok ? k.a_lp : 0.f);
 }
 
 template <int DT>
@@ -122,21 +127,33 @@ __global__ void __launch_bounds__(kThreads) backward_kernel(const BwdParams p) {
         const int vi = j * kThreads + threadIdx.x;
         if (vi >= nvec) continue;
         const int i0 = e0 + vi * kVecE;
-        uint4 o;
-        if (DT == 0) {
-          float g[4];
+        float g[kVecE];
+        {
           const uint32_t w[4] = {v[j].x, v[j].y, v[j].z, v[j].w};
 #pragma unroll
-          for (int q = 0; q < 4; ++q) g[q] = kind == 0 ? grad_entry(k, __uint_as_float(w[q]), i0 + q) : fill;
+          for (int q = 0; q < 4; ++q) {
+            if (DT == 0) {
+              g[q] = kind == 0 ? grad_entry_no_target(k, __uint_as_float(w[q])) : fill;
+            } else {
+              g[2 * q] = kind == 0 ? grad_entry_no_target(k, __uint_as_float(w[q] << 16)) : fill;
+              g[2 * q + 1] = kind == 0 ? grad_entry_no_target(k, __uint_as_float(w[q] & 0xFFFF0000u)) : fill;
+            }
+          }
+        }
+        if (kind == 0 && (unsigned)(k.tok - i0) < (unsigned)kVecE) {  // the vector that holds the target
+#pragma unroll
+          for (int q = 0; q < kVecE; ++q)
+            if (i0 + q == k.tok) g[q] += k.a_lp;
+        }
+        uint4 o;
+        if (DT == 0) {
           o = make_uint4(__float_as_uint(g[0]), __float_as_uint(g[1]), __float_as_uint(g[2]), __float_as_uint(g[3]));
         } else {
-          const uint32_t w[4] = {v[j].x, v[j].y, v[j].z, v[j].w};
           uint32_t r[4];
 #pragma unroll
           for (int q = 0; q < 4; ++q) {
-            const float g0 = kind == 0 ? grad_entry(k, __uint_as_float(w[q] << 16), i0 + 2 * q) : fill;
-            const float g1 = kind == 0 ? grad_entry(k, __uint_as_float(w[q] & 0xFFFF0000u), i0 + 2 * q + 1) : fill;
-            r[q] = (uint32_t)to_bf16_bits(g0) | ((uint32_t)to_bf16_bits(g1) << 16);
+            const __nv_bfloat162 h = __floats2bfloat162_rn(g[2 * q], g[2 * q + 1]);  // round to nearest even
+            r[q] = *reinterpret_cast<const uint32_t *>(&h);
           }
           o = make_uint4(r[0], r[1], r[2], r[3]);
         }
