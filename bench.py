@@ -265,6 +265,9 @@ def main():
             e3.e3_sample(ring[d % RING], temps, 0, d, row_base, args.sampler, out_tok=toks[d % RING],
                          out_logp=logp, out_ent=ent)
         e3.e3_token_logp_entropy(batch, all_toks, mask=mask, temp_scalar=1.0, out_logp=t_logp, out_ent=t_ent)
+        dz = torch.empty((ROWS, V), dtype=torch.bfloat16, device=dev)
+        e3.e3_token_logp_entropy_backward(batch[:ROWS], all_toks[:ROWS], t_logp[:ROWS], t_ent[:ROWS], t_logp[:ROWS],
+                                          t_ent[:ROWS], mask=mask[:ROWS], out=dz)
         torch.cuda.synchronize()
         print(json.dumps({"profile_launches": args.profile_launches}), flush=True)
         return

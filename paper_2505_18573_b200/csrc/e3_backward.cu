@@ -116,11 +116,18 @@ __global__ void __launch_bounds__(kThreads) backward_kernel(const BwdParams p) {
       const uint4 *src = reinterpret_cast<const uint4 *>(static_cast<const char *>(p.logits) +
                                                          (in0 + e0) * (DT == 0 ? 4 : 2));
       uint4 *dst = reinterpret_cast<uint4 *>(static_cast<char *>(p.dlogits) + (out0 + e0) * (DT == 0 ? 4 : 2));
+      if (kind != 0) {  // nothing to read: zeros or NaN
+        const uint32_t f1 = DT == 0 ? __float_as_uint(fill) : (kind == 1 ? 0u : 0x7FC07FC0u);
+        const uint4 o = make_uint4(f1, f1, f1, f1);
+        for (int vi = threadIdx.x; vi < nvec; vi += kThreads) __stcs(dst + vi, o);
+        for (int i = e0 + nvec * kVecE + threadIdx.x; i < e1; i += kThreads) store_grad<DT>(p.dlogits, out0 + i, fill);
+        continue;
+      }
       uint4 v[kPerThread];
 #pragma unroll
       for (int j = 0; j < kPerThread; ++j) {
         const int vi = j * kThreads + threadIdx.x;
-        if (kind == 0 && vi < nvec) v[j] = __ldcs(src + vi);
+        if (vi < nvec) v[j] = __ldcs(src + vi);
       }
 #pragma unroll
       for (int j = 0; j < kPerThread; ++j) {
@@ -133,14 +140,14 @@ __global__ void __launch_bounds__(kThreads) backward_kernel(const BwdParams p) {
 #pragma unroll
           for (int q = 0; q < 4; ++q) {
             if (DT == 0) {
-              g[q] = kind == 0 ? grad_entry_no_target(k, __uint_as_float(w[q])) : fill;
+              g[q] = grad_entry_no_target(k, __uint_as_float(w[q]));
             } else {
-              g[2 * q] = kind == 0 ? grad_entry_no_target(k, __uint_as_float(w[q] << 16)) : fill;
-              g[2 * q + 1] = kind == 0 ? grad_entry_no_target(k, __uint_as_float(w[q] & 0xFFFF0000u)) : fill;
+              g[2 * q] = grad_entry_no_target(k, __uint_as_float(w[q] << 16));
+              g[2 * q + 1] = grad_entry_no_target(k, __uint_as_float(w[q] & 0xFFFF0000u));
             }
           }
         }
-        if (kind == 0 && (unsigned)(k.tok - i0) < (unsigned)kVecE) {  // the vector that holds the target
+        if ((unsigned)(k.tok - i0) < (unsigned)kVecE) {  // the vector that holds the target
 #pragma unroll
           for (int q = 0; q < kVecE; ++q)
             if (i0 + q == k.tok) g[q] += k.a_lp;
@@ -161,7 +168,7 @@ __global__ void __launch_bounds__(kThreads) backward_kernel(const BwdParams p) {
       }
       // entries behind the last full vector (the row's length need not be a multiple of the vector)
       for (int i = e0 + nvec * kVecE + threadIdx.x; i < e1; i += kThreads)
-        store_grad<DT>(p.dlogits, out0 + i, kind == 0 ? grad_entry(k, load_logit<DT>(p.logits, in0 + i), i) : fill);
+        store_grad<DT>(p.dlogits, out0 + i, grad_entry(k, load_logit<DT>(p.logits, in0 + i), i));
     } else {
       for (int i = e0 + threadIdx.x; i < e1; i += kThreads)
         store_grad<DT>(p.dlogits, out0 + i, kind == 0 ? grad_entry(k, load_logit<DT>(p.logits, in0 + i), i) : fill);
