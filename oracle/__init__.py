@@ -199,6 +199,37 @@ def allocate_budget(k, G: int, G_min: int, G_max: int, greedy_mode: int = 0) -> 
     return out
 
 
+def difficulty_accumulate(n_c: np.ndarray, r_c: np.ndarray, question_ids, G, rewards) -> None:
+    """Adds one batch to the cumulative counts (int64) and rewards (float64), in place."""
+    assert n_c.dtype == np.int64 and r_c.dtype == np.float64 and n_c.size == r_c.size
+    q = np.ascontiguousarray(question_ids, dtype=np.int64)
+    g = np.ascontiguousarray(G, dtype=np.int32)
+    r = np.ascontiguousarray(rewards, dtype=np.float32)
+    assert r.size == int(g.sum())
+    rc = lib().e3o_difficulty_accumulate(C.c_int64(n_c.size), _p(n_c), _p(r_c), _p(q), _p(g), _p(r), C.c_int64(q.size))
+    if rc != 0:
+        raise ValueError("e3o_difficulty_accumulate: invalid argument")
+
+
+def difficulty_rank(n_c: np.ndarray, r_c: np.ndarray) -> np.ndarray:
+    n_c = np.ascontiguousarray(n_c, dtype=np.int64)
+    r_c = np.ascontiguousarray(r_c, dtype=np.float64)
+    out = np.empty(n_c.size, np.float64)
+    rc = lib().e3o_difficulty_rank(C.c_int64(n_c.size), _p(n_c), _p(r_c), _p(out))
+    if rc != 0:
+        raise ValueError("e3o_difficulty_rank: invalid argument")
+    return out
+
+
+def budget_curriculum(G: int, step: int, G_min_limit: int, G_max_limit: int, epochs_done: int):
+    lo, hi = C.c_int32(), C.c_int32()
+    rc = lib().e3o_budget_curriculum(C.c_int32(G), C.c_int32(step), C.c_int32(G_min_limit), C.c_int32(G_max_limit),
+                                     C.c_int64(epochs_done), C.byref(lo), C.byref(hi))
+    if rc != 0:
+        raise ValueError("e3o_budget_curriculum: invalid argument")
+    return lo.value, hi.value
+
+
 class Sched(C.Structure):
     _fields_ = [("tau", C.c_double), ("H_init", C.c_double), ("t", C.c_int64), ("t_anneal", C.c_int64),
                 ("t_max", C.c_int64), ("eta", C.c_double), ("V", C.c_int64), ("tau_min", C.c_double),

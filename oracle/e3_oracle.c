@@ -31,6 +31,7 @@
  *   Sec. 4.2 (H_init, H_t: average entropy of a batch)         -> e3o_masked_mean_entropy
  *   Eq. "adv" (Sec. 3.1)                                       -> e3o_group_advantage
  *   Algorithm 1 (Sec. 4.1)                                     -> e3o_allocate_budget
+ *   Sec. 4.1 difficulty model, G_min/G_max curriculum          -> e3o_difficulty_*, e3o_budget_curriculum
  *   Eq. "tp_adj" and the annealing equation (Sec. 4.2)         -> e3o_update_temperature
  */
 #define _GNU_SOURCE
@@ -578,3 +579,62 @@ int e3o_update_temperature(e3o_sched *s, double H_t, double *tau_next) {
   *tau_next = tau;
   return 0;
 }
+
+/* ------------------------------------------------------------------------- */
+/* Sec. 4.1, difficulty model.  For every question q_i of the dataset its      */
+/* cumulative rollout count n_i^c and cumulative reward r_i^c are recorded;    */
+/* at the end of a dataset iteration the questions are ranked by their         */
+/* average reward r_i^c / n_i^c in DESCENDING order (rank 1 = highest average  */
+/* reward = easiest) and k_i = rank(q_i) / |D|, so a larger k_i means a harder */
+/* question.  Readings where the paper is silent: equal averages keep dataset  */
+/* order (the earlier question gets the smaller rank); a question that was     */
+/* never rolled out has average reward 0.                                      */
+/* Pins: brute-force ranking with a library sort; k is a permutation of        */
+/* {1/|D|, ..., 1}; a harder question never has a smaller k.                    */
+/* ------------------------------------------------------------------------- */
+int e3o_difficulty_accumulate(int64_t D, int64_t *n_c, double *r_c, const int64_t *question_ids,
+                              const int32_t *G, const float *rewards, int64_t B) {
+  if (D < 0 || B < 0) return 1;
+  int64_t pos = 0;
+  for (int64_t b = 0; b < B; ++b) {
+    if (question_ids[b] < 0 || question_ids[b] >= D || G[b] < 0) return 1;
+    for (int32_t j = 0; j < G[b]; ++j) r_c[question_ids[b]] += (double)rewards[pos + j];
+    n_c[question_ids[b]] += G[b];
+    pos += G[b];
+  }
+  return 0;
+}
+
+int e3o_difficulty_rank(int64_t D, const int64_t *n_c, const double *r_c, double *out_k) {
+  if (D < 0) return 1;
+  for (int64_t i = 0; i < D; ++i) {
+    double ai = n_c[i] > 0 ? r_c[i] / (double)n_c[i] : 0.0;
+    int64_t rank = 1; /* 1 + number of questions that come before q_i in the descending order */
+    for (int64_t j = 0; j < D; ++j) {
+      if (j == i) continue;
+      double aj = n_c[j] > 0 ? r_c[j] / (double)n_c[j] : 0.0;
+      if (aj > ai || (aj == ai && j < i)) ++rank;
+    }
+    out_k[i] = (double)rank / (double)D;
+  }
+  return 0;
+}
+
+/* Sec. 4.1 / Sec. 5.2: G_min and G_max start at G; after each iteration of the   */
+/* dataset G_max grows and G_min shrinks by `step` (2 in the paper's runs) until  */
+/* the predefined limits are reached.  `epochs_done` = completed iterations.      */
+/* Pins: the paper's setting G = 8, step 2: (8,8), (6,10), (4,12), ...; limits.   */
+int e3o_budget_curriculum(int32_t G, int32_t step, int32_t G_min_limit, int32_t G_max_limit, int64_t epochs_done,
+                          int32_t *G_min, int32_t *G_max) {
+  if (G < 0 || step < 0 || epochs_done < 0 || G_min_limit < 0 || G_min_limit > G || G_max_limit < G) return 1;
+  int64_t lo = (int64_t)G, hi = (int64_t)G;
+  for (int64_t e = 0; e < epochs_done; ++e) {
+    if (hi + step <= G_max_limit) hi += step; else hi = G_max_limit;
+    if (lo - step >= G_min_limit) lo -= step; else lo = G_min_limit;
+    if (hi == G_max_limit && lo == G_min_limit) break;
+  }
+  *G_min = (int32_t)lo;
+  *G_max = (int32_t)hi;
+  return 0;
+}
+

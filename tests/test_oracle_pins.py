@@ -595,3 +595,44 @@ def test_backward_sums_to_zero_and_matches_autograd(oracle_mod):
     # out-of-range target and invalid temperature
     bad = o.token_logp_entropy_backward(z[:1], np.array([V], np.int32), g_lp[:1], g_en[:1])
     assert np.isnan(bad).all()
+
+
+# ----------------------------------------------------------------------------------------------
+# difficulty model and G_min / G_max curriculum (Sec. 4.1, Sec. 5.2)
+# ----------------------------------------------------------------------------------------------
+def test_difficulty_rank_against_a_library_sort_and_by_hand(oracle_mod):
+    o = oracle_mod
+    # by hand: averages 0.5, 1.0, 0.0, 0.5 -> descending order q1, q0, q3, q2 -> ranks 2, 1, 4, 3 (tie: earlier first)
+    k = o.difficulty_rank(np.array([4, 2, 8, 2]), np.array([2.0, 2.0, 0.0, 1.0]))
+    assert list(k) == [2 / 4, 1 / 4, 4 / 4, 3 / 4]
+    rng = np.random.default_rng(3)
+    D = 500
+    n = rng.integers(0, 40, size=D)                      # some questions never rolled out: average 0
+    r = np.floor(rng.random(D) * (n + 1)).astype(np.float64)
+    k = o.difficulty_rank(n, r)
+    avg = np.where(n > 0, r / np.maximum(n, 1), 0.0)
+    order = np.argsort(-avg, kind="stable")              # library routine: descending, stable
+    expect = np.empty(D); expect[order] = np.arange(1, D + 1) / D
+    assert np.array_equal(k, expect)
+    assert sorted(k) == [(i + 1) / D for i in range(D)]  # a permutation of 1/D ... 1
+    harder = avg[:, None] < avg[None, :]                 # i strictly harder than j -> k_i > k_j
+    assert np.all((k[:, None] > k[None, :])[harder])
+
+
+def test_difficulty_accumulate_adds_counts_and_rewards(oracle_mod):
+    o = oracle_mod
+    n = np.zeros(5, np.int64); r = np.zeros(5, np.float64)
+    o.difficulty_accumulate(n, r, [3, 0, 3], [2, 3, 1], [1, 0, 1, 1, 1, 0])
+    assert list(n) == [3, 0, 0, 3, 0] and list(r) == [3.0, 0.0, 0.0, 1.0, 0.0]
+    with pytest.raises(ValueError):
+        o.difficulty_accumulate(n, r, [5], [1], [1.0])
+
+
+def test_curriculum_follows_the_papers_setting(oracle_mod):
+    o = oracle_mod
+    # G = 8, +-2 per epoch (Sec. 5.2), limits 2 and 16
+    assert [o.budget_curriculum(8, 2, 2, 16, e) for e in range(6)] == [(8, 8), (6, 10), (4, 12), (2, 14), (2, 16), (2, 16)]
+    assert o.budget_curriculum(8, 2, 5, 9, 1) == (6, 9) and o.budget_curriculum(8, 2, 5, 9, 2) == (5, 9)
+    assert o.budget_curriculum(8, 0, 2, 16, 10) == (8, 8)
+    with pytest.raises(ValueError):
+        o.budget_curriculum(8, 2, 9, 16, 1)
