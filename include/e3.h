@@ -225,6 +225,33 @@ E3_API e3_status e3_group_advantage(const float *rewards, const int64_t *group_o
 E3_API e3_status e3_allocate_budget(const double *k, int64_t B, int32_t G, int32_t G_min, int32_t G_max,
                              int greedy_mode, int32_t *out_G);
 
+/*
+ * Difficulty model of Sec. 4.1, host only.  For every question of the dataset (D of them) the caller
+ * keeps the cumulative rollout count n_c[i] and the cumulative reward r_c[i] (plain arrays it owns,
+ * zero at the start of training; they are the whole state and can be stored as they are).
+ *
+ * e3_difficulty_accumulate adds one batch: question question_ids[b] was rolled out G[b] times and
+ * rewards holds those sum(G) rewards, group after group (the layout of e3_group_advantage).
+ * Nothing is changed when an argument is rejected (id outside [0, D), negative G).
+ *
+ * e3_difficulty_rank, called at the end of an iteration over the dataset, ranks the questions by their
+ * average reward r_c[i] / n_c[i] in descending order and writes k[i] = rank(q_i) / D: the question with
+ * the highest average reward gets 1/D, the hardest gets 1.  Equal averages keep dataset order; a question
+ * that was never rolled out counts as average reward 0.  out_k feeds e3_allocate_budget.
+ */
+E3_API e3_status e3_difficulty_accumulate(int64_t D, int64_t *n_c, double *r_c, const int64_t *question_ids,
+                                   const int32_t *G, const float *rewards, int64_t B);
+E3_API e3_status e3_difficulty_rank(int64_t D, const int64_t *n_c, const double *r_c, double *out_k);
+
+/*
+ * Curriculum on the budget bounds (Sec. 4.1, settings of Sec. 5.2): G_min = G_max = G at the start; after
+ * every finished iteration over the dataset G_max grows and G_min shrinks by `step` (2 in the paper's runs)
+ * until G_max_limit / G_min_limit.  epochs_done = number of finished iterations.  Host only.
+ * E3_ERR_INFEASIBLE unless G_min_limit <= G <= G_max_limit.
+ */
+E3_API e3_status e3_budget_curriculum(int32_t G, int32_t step, int32_t G_min_limit, int32_t G_max_limit,
+                               int64_t epochs_done, int32_t *G_min, int32_t *G_max);
+
 /* Scheduler state, owned by the caller; plain data, can be copied or stored as is. */
 typedef struct {
   double tau;      /* current temperature tau_t (> 0) */

@@ -24,7 +24,7 @@ E3_SAMPLE_BLOCK = 256
 EXPORTS = ("e3_status_string", "e3_workspace_bytes", "e3_sample", "e3_token_logp_entropy",
            "e3_token_logp_entropy_backward",
            "e3_masked_mean_entropy", "e3_masked_mean_entropy_static", "e3_group_advantage", "e3_allocate_budget", "e3_update_temperature",
-           "e3_anneal_target")
+           "e3_anneal_target", "e3_difficulty_accumulate", "e3_difficulty_rank", "e3_budget_curriculum")
 
 
 class E3Error(RuntimeError):
@@ -79,6 +79,14 @@ def lib() -> C.CDLL:
         L.e3_allocate_budget.argtypes = [C.c_void_p, C.c_int64, C.c_int32, C.c_int32, C.c_int32, C.c_int, C.c_void_p]
         L.e3_update_temperature.restype = C.c_int
         L.e3_update_temperature.argtypes = [C.POINTER(e3_sched), C.c_double, C.POINTER(C.c_double)]
+        L.e3_difficulty_accumulate.restype = C.c_int
+        L.e3_difficulty_accumulate.argtypes = [C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                                               C.c_int64]
+        L.e3_difficulty_rank.restype = C.c_int
+        L.e3_difficulty_rank.argtypes = [C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p]
+        L.e3_budget_curriculum.restype = C.c_int
+        L.e3_budget_curriculum.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int64,
+                                           C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
         L.e3_anneal_target.restype = C.c_double
         L.e3_anneal_target.argtypes = [C.POINTER(e3_sched)]
         _lib = L
@@ -304,3 +312,38 @@ def e3_update_temperature(s: e3_sched, H_t: float) -> float:
 
 def e3_anneal_target(s: e3_sched) -> float:
     return float(lib().e3_anneal_target(C.byref(s)))
+
+
+def e3_difficulty_accumulate(n_c, r_c, question_ids, G, rewards) -> None:
+    """Adds one batch to the caller's cumulative counts (numpy int64) and rewards (numpy float64), in place."""
+    import numpy as np
+    if n_c.dtype != np.int64 or r_c.dtype != np.float64 or n_c.size != r_c.size:
+        raise ValueError("n_c must be int64 and r_c float64, one entry per question")
+    q = np.ascontiguousarray(question_ids, dtype=np.int64)
+    g = np.ascontiguousarray(G, dtype=np.int32)
+    r = np.ascontiguousarray(rewards, dtype=np.float32)
+    if g.size != q.size or r.size != int(g.sum()):
+        raise ValueError("one G per question id and sum(G) rewards are needed")
+    st = lib().e3_difficulty_accumulate(n_c.size, n_c.ctypes.data, r_c.ctypes.data, q.ctypes.data, g.ctypes.data,
+                                        r.ctypes.data, q.size)
+    _check("e3_difficulty_accumulate", st)
+
+
+def e3_difficulty_rank(n_c, r_c):
+    """Normalised difficulty ranks k (numpy float64, one per question) from the cumulative statistics."""
+    import numpy as np
+    n = np.ascontiguousarray(n_c, dtype=np.int64)
+    r = np.ascontiguousarray(r_c, dtype=np.float64)
+    out = np.empty(n.size, np.float64)
+    st = lib().e3_difficulty_rank(n.size, n.ctypes.data, r.ctypes.data, out.ctypes.data)
+    _check("e3_difficulty_rank", st)
+    return out
+
+
+def e3_budget_curriculum(G: int, step: int, G_min_limit: int, G_max_limit: int, epochs_done: int):
+    """(G_min, G_max) after ``epochs_done`` finished iterations over the dataset."""
+    lo, hi = C.c_int32(), C.c_int32()
+    st = lib().e3_budget_curriculum(G, step, G_min_limit, G_max_limit, epochs_done, C.byref(lo), C.byref(hi))
+    _check("e3_budget_curriculum", st)
+    return lo.value, hi.value
+

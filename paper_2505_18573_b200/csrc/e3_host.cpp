@@ -100,3 +100,53 @@ extern "C" e3_status e3_update_temperature(e3_sched *s, double H_t, double *tau_
   *tau_next = tau;
   return E3_OK;
 }
+
+// ---------------------------------------------------------------------------------------------
+// Sec. 4.1 difficulty model and the G_min / G_max curriculum
+// ---------------------------------------------------------------------------------------------
+extern "C" e3_status e3_difficulty_accumulate(int64_t D, int64_t *n_c, double *r_c, const int64_t *question_ids,
+                                              const int32_t *G, const float *rewards, int64_t B) {
+  if (D < 0 || B < 0 || (D > 0 && (!n_c || !r_c)) || (B > 0 && (!question_ids || !G))) return E3_ERR_INVALID_ARG;
+  int64_t total = 0;
+  for (int64_t b = 0; b < B; ++b) {  // look at everything before touching the state
+    if (question_ids[b] < 0 || question_ids[b] >= D || G[b] < 0) return E3_ERR_INVALID_ARG;
+    total += G[b];
+  }
+  if (total > 0 && !rewards) return E3_ERR_INVALID_ARG;
+  const float *r = rewards;
+  for (int64_t b = 0; b < B; ++b) {
+    double sum = 0.0;
+    for (int32_t j = 0; j < G[b]; ++j) sum += static_cast<double>(r[j]);
+    r += G[b];
+    r_c[question_ids[b]] += sum;
+    n_c[question_ids[b]] += G[b];
+  }
+  return E3_OK;
+}
+
+extern "C" e3_status e3_difficulty_rank(int64_t D, const int64_t *n_c, const double *r_c, double *out_k) {
+  if (D < 0 || (D > 0 && (!n_c || !r_c || !out_k))) return E3_ERR_INVALID_ARG;
+  std::vector<double> avg(static_cast<size_t>(D));
+  for (int64_t i = 0; i < D; ++i) {
+    if (n_c[i] < 0 || !std::isfinite(r_c[i])) return E3_ERR_INVALID_ARG;
+    avg[i] = n_c[i] > 0 ? r_c[i] / static_cast<double>(n_c[i]) : 0.0;
+  }
+  std::vector<int64_t> order(static_cast<size_t>(D));
+  std::iota(order.begin(), order.end(), int64_t(0));
+  std::stable_sort(order.begin(), order.end(), [&](int64_t a, int64_t b) { return avg[a] > avg[b]; });
+  for (int64_t pos = 0; pos < D; ++pos) out_k[order[pos]] = static_cast<double>(pos + 1) / static_cast<double>(D);
+  return E3_OK;
+}
+
+extern "C" e3_status e3_budget_curriculum(int32_t G, int32_t step, int32_t G_min_limit, int32_t G_max_limit,
+                                          int64_t epochs_done, int32_t *G_min, int32_t *G_max) {
+  if (!G_min || !G_max || G < 0 || step < 0 || epochs_done < 0 || G_min_limit < 0) return E3_ERR_INVALID_ARG;
+  if (G_min_limit > G || G_max_limit < G) return E3_ERR_INFEASIBLE;
+  // closed form of "widen by `step` per finished epoch until the limit"
+  const int64_t moved = static_cast<int64_t>(step) * epochs_done;  // step, epochs_done >= 0
+  const int64_t up = static_cast<int64_t>(G_max_limit) - G, down = static_cast<int64_t>(G) - G_min_limit;
+  *G_max = static_cast<int32_t>(G + (step > 0 && epochs_done > up / step ? up : std::min(moved, up)));
+  *G_min = static_cast<int32_t>(G - (step > 0 && epochs_done > down / step ? down : std::min(moved, down)));
+  return E3_OK;
+}
+

@@ -118,3 +118,42 @@ def test_update_temperature_matches_oracle(e3):
     with pytest.raises(e3.E3Error):
         e3.e3_update_temperature(s, 1e3)
     assert s.tau == 4.0 and s.t == 0
+
+
+def test_difficulty_model_and_curriculum_match_the_oracle(oracle_mod):
+    """Sec. 4.1: cumulative statistics, descending-average-reward ranks, bounds curriculum; then Algorithm 1 on the ranks."""
+    import numpy as np
+    from paper_2505_18573_b200 import binding as e3
+    o = oracle_mod
+    rng = np.random.default_rng(11)
+    D, B = 300, 64
+    n1 = np.zeros(D, np.int64); r1 = np.zeros(D, np.float64)
+    n2 = np.zeros(D, np.int64); r2 = np.zeros(D, np.float64)
+    p_q = rng.random(D)
+    for epoch in range(3):
+        g_min, g_max = e3.e3_budget_curriculum(8, 2, 2, 16, epoch)
+        assert (g_min, g_max) == o.budget_curriculum(8, 2, 2, 16, epoch)
+        k = e3.e3_difficulty_rank(n1, r1)
+        assert np.array_equal(k, o.difficulty_rank(n2, r2))
+        for start in range(0, D - B + 1, B):
+            ids = np.arange(start, start + B)
+            G = e3.e3_allocate_budget(k[ids], 8, g_min, g_max)
+            assert sum(G) == 8 * B and G == list(o.allocate_budget(k[ids], 8, g_min, g_max))
+            rewards = (rng.random(sum(G)) < np.repeat(p_q[ids], G)).astype(np.float32)
+            e3.e3_difficulty_accumulate(n1, r1, ids, G, rewards)
+            o.difficulty_accumulate(n2, r2, ids, G, rewards)
+            assert np.array_equal(n1, n2) and np.array_equal(r1, r2)
+    k = e3.e3_difficulty_rank(n1, r1)
+    assert sorted(k) == [(i + 1) / D for i in range(D)]
+    seen = n1 > 0
+    assert np.corrcoef(k[seen], p_q[seen])[0, 1] < -0.8          # easy questions (high success rate) get small k
+    for e in range(12):
+        assert e3.e3_budget_curriculum(8, 3, 1, 20, e) == o.budget_curriculum(8, 3, 1, 20, e)
+    L = e3.lib()
+    assert L.e3_budget_curriculum(8, 2, 9, 16, 1, None, None) == 1
+    n3 = np.zeros(4, np.int64); r3 = np.zeros(4, np.float64)
+    with pytest.raises(e3.E3Error):
+        e3.e3_difficulty_accumulate(n3, r3, [1, 4], [1, 1], [1.0, 1.0])
+    assert n3.sum() == 0 and r3.sum() == 0                        # a rejected batch changes nothing
+    with pytest.raises(e3.E3Error):
+        e3.e3_budget_curriculum(8, 2, 9, 16, 1)
