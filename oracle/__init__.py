@@ -199,6 +199,24 @@ def allocate_budget(k, G: int, G_min: int, G_max: int, greedy_mode: int = 0) -> 
     return out
 
 
+def grpo_objective(logp, logp_old, mask, adv, group_offsets, clip_eps: float = 0.2):
+    """Returns (J, grad float64 [n_seq, seq_len], clipped fraction).  logp arrays are [n_seq, seq_len]."""
+    logp = np.ascontiguousarray(logp, dtype=np.float32)
+    logp_old = np.ascontiguousarray(logp_old, dtype=np.float32)
+    n_seq, seq_len = logp.shape
+    mask = None if mask is None else np.ascontiguousarray(mask, dtype=np.uint8).reshape(n_seq, seq_len)
+    adv = np.ascontiguousarray(adv, dtype=np.float32)
+    off = np.ascontiguousarray(group_offsets, dtype=np.int64)
+    grad = np.empty((n_seq, seq_len), np.float64)
+    J, frac = C.c_double(), C.c_double()
+    rc = lib().e3o_grpo_objective(_p(logp), _p(logp_old), _p(mask), C.c_int64(n_seq), C.c_int64(seq_len), _p(adv),
+                                  _p(off), C.c_int64(off.size - 1), C.c_float(clip_eps), _p(grad), C.byref(J),
+                                  C.byref(frac))
+    if rc != 0:
+        raise ValueError("e3o_grpo_objective: invalid argument")
+    return J.value, grad, frac.value
+
+
 def difficulty_accumulate(n_c: np.ndarray, r_c: np.ndarray, question_ids, G, rewards) -> None:
     """Adds one batch to the cumulative counts (int64) and rewards (float64), in place."""
     assert n_c.dtype == np.int64 and r_c.dtype == np.float64 and n_c.size == r_c.size

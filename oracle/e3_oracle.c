@@ -30,6 +30,7 @@
  *             through the softmax of App. A)                   -> e3o_token_logp_entropy_backward
  *   Sec. 4.2 (H_init, H_t: average entropy of a batch)         -> e3o_masked_mean_entropy
  *   Eq. "adv" (Sec. 3.1)                                       -> e3o_group_advantage
+ *   GRPO objective (Sec. 3.1, no KL term)                      -> e3o_grpo_objective
  *   Algorithm 1 (Sec. 4.1)                                     -> e3o_allocate_budget
  *   Sec. 4.1 difficulty model, G_min/G_max curriculum          -> e3o_difficulty_*, e3o_budget_curriculum
  *   Eq. "tp_adj" and the annealing equation (Sec. 4.2)         -> e3o_update_temperature
@@ -635,6 +636,61 @@ int e3o_budget_curriculum(int32_t G, int32_t step, int32_t G_min_limit, int32_t 
   }
   *G_min = (int32_t)lo;
   *G_max = (int32_t)hi;
+  return 0;
+}
+
+/* ------------------------------------------------------------------------- */
+/* The GRPO objective of Sec. 3.1 without the KL term (the paper drops it):    */
+/*   J = mean over questions q of                                              */
+/*         (1/G_q) sum_{i in group q} (1/|o_i|) sum_{t=1..|o_i|}               */
+/*           min( r_{i,t} A_i , clip(r_{i,t}, 1-eps, 1+eps) A_i ),             */
+/*   r_{i,t} = pi_theta(o_{i,t}) / pi_theta_old(o_{i,t}) = exp(logp - logp_old).*/
+/* Tokens are laid out [n_seq, seq_len]; mask marks the |o_i| response tokens  */
+/* of sequence i; A_i is the group-relative advantage of response i (Eq. adv),  */
+/* the same for all its tokens; groups are runs of sequences given by offsets   */
+/* (their sizes G_q differ under the dynamic rollout budget).  A response       */
+/* without tokens contributes 0 but still counts in G_q.                        */
+/* Also returns dJ/dlogp per token (0 where the clipped branch is the smaller    */
+/* one, i.e. A > 0 and r > 1+eps, or A < 0 and r < 1-eps; 0 on masked tokens)    */
+/* and the fraction of response tokens where that happened.                     */
+/* Pins: logp == logp_old gives J = mean_q mean_i A_i; hand cases of the clip;   */
+/* central differences of J; an autograd library.                               */
+/* ------------------------------------------------------------------------- */
+int e3o_grpo_objective(const float *logp, const float *logp_old, const uint8_t *mask, int64_t n_seq,
+                       int64_t seq_len, const float *adv, const int64_t *group_offsets, int64_t n_groups,
+                       float clip_eps, double *out_grad /* [n_seq*seq_len] or NULL */, double *out_J,
+                       double *out_clip_frac) {
+  if (n_seq < 0 || seq_len < 0 || n_groups < 0 || !(clip_eps >= 0.0f)) return 1;
+  if (n_groups > 0 && (group_offsets[0] != 0 || group_offsets[n_groups] != n_seq)) return 1;
+  double J = 0.0, clipped = 0.0, tokens = 0.0;
+  double lo = 1.0 - (double)clip_eps, hi = 1.0 + (double)clip_eps;
+  for (int64_t q = 0; q < n_groups; ++q) {
+    int64_t a = group_offsets[q], b = group_offsets[q + 1];
+    if (b < a) return 1;
+    double Gq = (double)(b - a), Jq = 0.0;
+    for (int64_t i = a; i < b; ++i) {
+      double len = 0.0;
+      for (int64_t t = 0; t < seq_len; ++t) len += (!mask || mask[i * seq_len + t]) ? 1.0 : 0.0;
+      double A = (double)adv[i], Ji = 0.0;
+      for (int64_t t = 0; t < seq_len; ++t) {
+        int64_t j = i * seq_len + t;
+        if (out_grad) out_grad[j] = 0.0;
+        if (mask && !mask[j]) continue;
+        double r = exp((double)logp[j] - (double)logp_old[j]);
+        double rc = r < lo ? lo : (r > hi ? hi : r);
+        double s1 = r * A, s2 = rc * A;
+        int clip_active = s2 < s1; /* the clipped term is the strictly smaller one: no gradient */
+        Ji += clip_active ? s2 : s1;
+        tokens += 1.0;
+        clipped += clip_active ? 1.0 : 0.0;
+        if (out_grad) out_grad[j] = clip_active ? 0.0 : s1 / (len * Gq * (double)n_groups);
+      }
+      if (len > 0.0) Jq += Ji / len;
+    }
+    if (Gq > 0.0) J += Jq / Gq;
+  }
+  *out_J = n_groups > 0 ? J / (double)n_groups : 0.0;
+  if (out_clip_frac) *out_clip_frac = tokens > 0.0 ? clipped / tokens : 0.0;
   return 0;
 }
 

@@ -636,3 +636,79 @@ def test_curriculum_follows_the_papers_setting(oracle_mod):
     assert o.budget_curriculum(8, 0, 2, 16, 10) == (8, 8)
     with pytest.raises(ValueError):
         o.budget_curriculum(8, 2, 9, 16, 1)
+
+
+# ----------------------------------------------------------------------------------------------
+# GRPO objective (Sec. 3.1, no KL term)
+# ----------------------------------------------------------------------------------------------
+def _grpo_case(seed=0, n_groups=5, seq_len=12):
+    rng = np.random.default_rng(seed)
+    sizes = rng.integers(1, 5, size=n_groups)
+    off = np.concatenate([[0], np.cumsum(sizes)]).astype(np.int64)
+    n_seq = int(off[-1])
+    lengths = rng.integers(0, seq_len + 1, size=n_seq)
+    lengths[0] = 0                                                     # a response without tokens
+    mask = (np.arange(seq_len)[None, :] < lengths[:, None]).astype(np.uint8)
+    logp_old = -rng.random((n_seq, seq_len)).astype(np.float32) * 3
+    logp = (logp_old + rng.normal(size=(n_seq, seq_len)).astype(np.float32) * 0.3).astype(np.float32)
+    adv = rng.normal(size=n_seq).astype(np.float32)
+    return logp, logp_old, mask, adv, off
+
+
+def test_grpo_objective_hand_cases(oracle_mod):
+    o = oracle_mod
+    ln = np.log
+    # one question, two responses of 2 and 1 tokens, eps = 0.2
+    logp_old = np.zeros((2, 2), np.float32)
+    logp = np.array([[ln(1.5), ln(0.5)], [ln(1.1), 0.0]], np.float32)
+    mask = np.array([[1, 1], [1, 0]], np.uint8)
+    adv = np.array([1.0, -2.0], np.float32)
+    J, g, frac = o.grpo_objective(logp, logp_old, mask, adv, [0, 2], 0.2)
+    # response 0 (A = 1): r = 1.5 -> min(1.5, 1.2) = 1.2 (clipped, no gradient); r = 0.5 -> min(0.5, 0.8) = 0.5
+    # response 1 (A = -2): r = 1.1 -> min(-2.2, -2.2) = -2.2
+    assert J == pytest.approx(0.5 * ((1.2 + 0.5) / 2 + (-2.2) / 1), abs=1e-6)
+    assert g[0, 0] == 0.0 and g[0, 1] == pytest.approx(0.5 * 1.0 / (2 * 2), abs=1e-7)
+    assert g[1, 0] == pytest.approx(1.1 * -2.0 / (1 * 2), abs=1e-6) and g[1, 1] == 0.0
+    assert frac == pytest.approx(1 / 3)
+    # negative advantage, ratio below the range: the clipped term (0.8 A) is smaller than r A: no gradient
+    J2, g2, _ = o.grpo_objective(np.full((1, 1), ln(0.5), np.float32), np.zeros((1, 1), np.float32), None,
+                                 np.array([-1.0], np.float32), [0, 1], 0.2)
+    assert J2 == pytest.approx(-0.8, abs=1e-6) and g2[0, 0] == 0.0
+
+
+def test_grpo_objective_at_the_old_policy_is_the_mean_advantage(oracle_mod):
+    o = oracle_mod
+    logp, logp_old, mask, adv, off = _grpo_case(1)
+    J, g, frac = o.grpo_objective(logp_old, logp_old, mask, adv, off, 0.2)
+    adv = adv.astype(np.float64)
+    has = mask.sum(axis=1) > 0
+    expect = np.mean([np.sum(adv[off[q]:off[q + 1]][has[off[q]:off[q + 1]]]) / (off[q + 1] - off[q]) for q in range(off.size - 1)])
+    assert J == pytest.approx(expect, abs=1e-9) and frac == 0.0
+    w = 1.0 / (np.maximum(mask.sum(axis=1), 1) * np.repeat(np.diff(off), np.diff(off)) * (off.size - 1))
+    assert np.allclose(g, mask * (adv * w)[:, None], atol=1e-12)
+
+
+def test_grpo_objective_gradient_against_central_differences_and_autograd(oracle_mod):
+    import torch
+    o = oracle_mod
+    logp, logp_old, mask, adv, off = _grpo_case(2)
+    J, g, _ = o.grpo_objective(logp, logp_old, mask, adv, off, 0.2)
+    r = np.exp(logp.astype(np.float64) - logp_old)
+    h = 2.0 ** -10
+    for (i, t) in [(1, 0), (2, 3), (5, 1), (7, 0)]:
+        if not mask[i, t] or min(abs(r[i, t] - 0.8), abs(r[i, t] - 1.2)) < 0.02:
+            continue                                                   # off the response or next to a kink
+        lp, lm = logp.copy(), logp.copy()
+        lp[i, t] += h; lm[i, t] -= h
+        num = (o.grpo_objective(lp, logp_old, mask, adv, off, 0.2)[0] - o.grpo_objective(lm, logp_old, mask, adv, off, 0.2)[0]) / (2 * h)
+        assert g[i, t] == pytest.approx(num, abs=1e-6)
+    x = torch.tensor(logp, dtype=torch.float64, requires_grad=True)
+    ratio = torch.exp(x - torch.tensor(logp_old, dtype=torch.float64))
+    A = torch.tensor(adv, dtype=torch.float64)[:, None]
+    eps = float(np.float32(0.2))
+    sur = torch.minimum(ratio * A, torch.clamp(ratio, 1 - eps, 1 + eps) * A) * torch.tensor(mask, dtype=torch.float64)
+    per_seq = sur.sum(dim=1) / torch.clamp(torch.tensor(mask.sum(axis=1), dtype=torch.float64), min=1)
+    Jt = sum(per_seq[off[q]:off[q + 1]].sum() / (off[q + 1] - off[q]) for q in range(off.size - 1)) / (off.size - 1)
+    Jt.backward()
+    assert J == pytest.approx(float(Jt), abs=1e-12)
+    assert np.abs(g - x.grad.numpy()).max() < 1e-12
