@@ -375,6 +375,15 @@ def main():
     bwd_us = time_alone(lambda d: e3.e3_token_logp_entropy_backward(ring[d % RING], targets1, logp, ent, g1, g1,
                                                                     temps=temps, out=dz))
 
+    # GRPO objective over 512 responses x 2,048 tokens (latency-bound: a few bytes per token)
+    gl = torch.randn((ROWS, 2048), device=dev) * 0.1 - 1.0
+    gmask, _ = inputs.response_mask(ROWS, 2048, seed=9, min_len=256, device=dev)
+    gout = torch.empty(2, dtype=torch.float64, device=dev)
+    ggrad = torch.empty((ROWS, 2048), dtype=torch.float32, device=dev)
+    gws = torch.empty(e3.e3_workspace_bytes(e3.E3_CALL_GRPO_OBJECTIVE, ROWS), dtype=torch.uint8, device=dev)
+    grpo_us = time_alone(lambda d: e3.e3_grpo_objective(gl, gl, adv, offsets, mask=gmask, out_g_logp=ggrad, out=gout,
+                                                        workspace=gws))
+
     if rank == 0:
         peak, peak_kind = _peaks()
         bytes_per_launch = ROWS * V * 2 + ROWS * 4 + ROWS * 12
@@ -399,6 +408,8 @@ def main():
                               "GBps_incl_small_kernels_and_sync": train_bytes / (ms_tail * 1e-3 / args.steps) / 1e9},
             "kernels": {k: {"us_per_launch": v, "GBps": bytes_per_launch / v / 1e3, "frac": bytes_per_launch / v / 1e3 / peak}
                         for k, v in alone.items()},
+            "grpo_objective": {"kernel": "e3_grpo_objective, 512 responses x 2,048 tokens (next row of the scope table)",
+                               "us_per_call": grpo_us},
             "backward": {"kernel": "e3_token_logp_entropy_backward (next row of the scope table, not part of the step)",
                          "us_per_launch": bwd_us, "GBps_read_plus_write": 2 * ROWS * V * 2 / bwd_us / 1e3,
                          "frac": 2 * ROWS * V * 2 / bwd_us / 1e3 / peak},

@@ -68,14 +68,16 @@ typedef enum {
 typedef enum {
   E3_CALL_SAMPLE = 0,
   E3_CALL_TOKEN_LOGP_ENTROPY = 1,
-  E3_CALL_MASKED_MEAN_ENTROPY = 2
+  E3_CALL_MASKED_MEAN_ENTROPY = 2,
+  E3_CALL_GRPO_OBJECTIVE = 3
 } e3_call;
 
 /* Human-readable name of a status code (static string). */
 E3_API const char *e3_status_string(e3_status s);
 
 /* Bytes of device scratch a call uses for the given problem size.  For
- * E3_CALL_MASKED_MEAN_ENTROPY `rows` is the number of tokens n and V, dt are ignored.
+ * E3_CALL_MASKED_MEAN_ENTROPY `rows` is the number of tokens n, for E3_CALL_GRPO_OBJECTIVE the number of
+ * responses n_seq; V, dt are ignored for both.
  * Scratch contents on entry never matter.  A workspace must not be shared by calls that can run
  * at the same time (different streams without ordering).  It must be 16-byte aligned. */
 E3_API size_t e3_workspace_bytes(e3_call which, int64_t rows, int64_t V, e3_dtype dt);
@@ -212,6 +214,34 @@ E3_API e3_status e3_masked_mean_entropy_static(const float *ent, const uint8_t *
  */
 E3_API e3_status e3_group_advantage(const float *rewards, const int64_t *group_offsets, int64_t n_groups,
                              float eps, int unbiased, float *out_adv, uint8_t *out_group_flags, void *stream);
+
+/*
+ * The GRPO objective of Sec. 3.1 without its KL term (the paper does not use it), over one batch:
+ *   J = mean over questions q of (1/G_q) sum_{i in q} (1/|o_i|) sum_{t <= |o_i|}
+ *         min( r_{i,t} A_i , clip(r_{i,t}, 1 - clip_eps, 1 + clip_eps) A_i ),
+ *   r_{i,t} = exp(logp[i,t] - logp_old[i,t]).
+ * Tokens are laid out [n_seq, seq_len]; mask marks the |o_i| response tokens of response i; adv[i] is the
+ * group-relative advantage of response i (e3_group_advantage), the same for all its tokens; question q
+ * owns the responses [group_offsets[q], group_offsets[q+1]) (sizes differ under the dynamic budget).  A
+ * response without tokens contributes 0 but counts in G_q.
+ *
+ *   logp, logp_old   device float [n_seq * seq_len] (e3_token_logp_entropy outputs of the current and the old policy)
+ *   mask             device uint8 [n_seq * seq_len] or NULL (= all ones)
+ *   adv              device float [n_seq];  group_offsets: device int64 [n_groups + 1], non-decreasing,
+ *                    [0] == 0, [n_groups] == n_seq (a response outside every group contributes nothing)
+ *   out_g_logp       NULL or device float [n_seq * seq_len]: dJ/dlogp per token; 0 on tokens outside the mask and
+ *                    where the clipped term is the smaller one (A > 0 and r > 1 + eps, or A < 0 and r < 1 - eps).
+ *                    This is the g_logp of e3_token_logp_entropy_backward (J is maximised: negate for a loss).
+ *   out_objective    device double scalar, required;  out_clip_frac: NULL or device double scalar, the fraction of
+ *                    response tokens whose clipped term is active
+ *   workspace        e3_workspace_bytes(E3_CALL_GRPO_OBJECTIVE, n_seq, 0, 0) bytes of device scratch, 8-byte aligned
+ * All arithmetic is fp64 in a fixed order: results are reproducible, and the clip decision does not depend
+ * on fp32 rounding.
+ */
+E3_API e3_status e3_grpo_objective(const float *logp, const float *logp_old, const uint8_t *mask, int64_t n_seq,
+                            int64_t seq_len, const float *adv, const int64_t *group_offsets, int64_t n_groups,
+                            float clip_eps, float *out_g_logp, double *out_objective, double *out_clip_frac,
+                            void *workspace, size_t workspace_bytes, void *stream);
 
 /*
  * Algorithm 1 (Dynamic Rollout Budget), host only.  k[i] in [0, 1] is the normalised difficulty

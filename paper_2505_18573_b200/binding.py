@@ -18,11 +18,11 @@ LIB_PATH = os.path.join(_PKG, "libe3.so")
 E3_OK = 0
 E3_F32, E3_BF16 = 0, 1
 E3_SAMPLER_TOKEN, E3_SAMPLER_BLOCK, E3_SAMPLER_TOKEN_AUDIT = 0, 1, 2
-E3_CALL_SAMPLE, E3_CALL_TOKEN_LOGP_ENTROPY, E3_CALL_MASKED_MEAN_ENTROPY = 0, 1, 2
+E3_CALL_SAMPLE, E3_CALL_TOKEN_LOGP_ENTROPY, E3_CALL_MASKED_MEAN_ENTROPY, E3_CALL_GRPO_OBJECTIVE = 0, 1, 2, 3
 E3_SAMPLE_BLOCK = 256
 
 EXPORTS = ("e3_status_string", "e3_workspace_bytes", "e3_sample", "e3_token_logp_entropy",
-           "e3_token_logp_entropy_backward",
+           "e3_token_logp_entropy_backward", "e3_grpo_objective",
            "e3_masked_mean_entropy", "e3_masked_mean_entropy_static", "e3_group_advantage", "e3_allocate_budget", "e3_update_temperature",
            "e3_anneal_target", "e3_difficulty_accumulate", "e3_difficulty_rank", "e3_budget_curriculum")
 
@@ -79,6 +79,10 @@ def lib() -> C.CDLL:
         L.e3_allocate_budget.argtypes = [C.c_void_p, C.c_int64, C.c_int32, C.c_int32, C.c_int32, C.c_int, C.c_void_p]
         L.e3_update_temperature.restype = C.c_int
         L.e3_update_temperature.argtypes = [C.POINTER(e3_sched), C.c_double, C.POINTER(C.c_double)]
+        L.e3_grpo_objective.restype = C.c_int
+        L.e3_grpo_objective.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_void_p, C.c_void_p,
+                                        C.c_int64, C.c_float, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t,
+                                        C.c_void_p]
         L.e3_difficulty_accumulate.restype = C.c_int
         L.e3_difficulty_accumulate.argtypes = [C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                                C.c_int64]
@@ -285,6 +289,35 @@ def e3_group_advantage(rewards, group_offsets, eps: float = 1e-6, unbiased: bool
                                   _ptr(out_adv), _ptr(out_flags), _stream(stream))
     _check("e3_group_advantage", st)
     return out_adv, out_flags
+
+
+def e3_grpo_objective(logp, logp_old, adv, group_offsets, mask=None, clip_eps: float = 0.2, out_g_logp=None,
+                      want_grad: bool = True, out=None, workspace=None, stream=None):
+    """GRPO objective over tokens laid out [n_seq, seq_len].  Returns (out float64 CUDA [2] = (J, clipped
+    fraction), g_logp float32 [n_seq, seq_len] | None)."""
+    for name, t in (("logp", logp), ("logp_old", logp_old), ("adv", adv), ("group_offsets", group_offsets), ("mask", mask)):
+        _dev(t, name)
+    if logp.dim() != 2 or logp.shape != logp_old.shape or not logp.is_contiguous() or not logp_old.is_contiguous():
+        raise ValueError("logp and logp_old must be contiguous [n_seq, seq_len] tensors of the same shape")
+    if logp.dtype != torch.float32 or logp_old.dtype != torch.float32 or adv.dtype != torch.float32:
+        raise ValueError("logp, logp_old and adv must be float32")
+    n_seq, seq_len = logp.shape
+    if adv.numel() != n_seq or group_offsets.dtype != torch.int64:
+        raise ValueError("adv needs one entry per response, group_offsets must be int64")
+    if mask is not None and (mask.dtype != torch.uint8 or mask.numel() != n_seq * seq_len or not mask.is_contiguous()):
+        raise ValueError("mask must be contiguous uint8 with one entry per token")
+    if out_g_logp is None and want_grad:
+        out_g_logp = torch.empty((n_seq, seq_len), dtype=torch.float32, device=logp.device)
+    if out is None:
+        out = torch.empty(2, dtype=torch.float64, device=logp.device)
+    need = e3_workspace_bytes(E3_CALL_GRPO_OBJECTIVE, n_seq)
+    if workspace is None:
+        workspace = torch.empty(need, dtype=torch.uint8, device=logp.device)
+    st = lib().e3_grpo_objective(_ptr(logp), _ptr(logp_old), _ptr(mask), n_seq, seq_len, _ptr(adv), _ptr(group_offsets),
+                                 group_offsets.numel() - 1, float(clip_eps), _ptr(out_g_logp), out.data_ptr(),
+                                 out.data_ptr() + 8, _ptr(workspace), workspace.numel(), _stream(stream))
+    _check("e3_grpo_objective", st)
+    return out, out_g_logp
 
 
 def e3_allocate_budget(k, G: int, G_min: int, G_max: int, greedy_mode: int = 0):

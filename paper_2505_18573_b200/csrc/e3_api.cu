@@ -6,6 +6,10 @@
 #include "e3_rows.cuh"
 #include "e3_small.cuh"
 
+namespace e3 {
+size_t grpo_workspace_bytes(int64_t n_seq);
+}
+
 namespace {
 
 inline bool misaligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) != 0; }
@@ -42,6 +46,7 @@ extern "C" size_t e3_workspace_bytes(e3_call which, int64_t rows, int64_t V, e3_
     case E3_CALL_SAMPLE: return e3::rows_workspace_bytes();
     case E3_CALL_TOKEN_LOGP_ENTROPY: return e3::rows_workspace_bytes();
     case E3_CALL_MASKED_MEAN_ENTROPY: return e3::mean_workspace_bytes(rows < 0 ? 0 : rows);
+    case E3_CALL_GRPO_OBJECTIVE: return e3::grpo_workspace_bytes(rows);
   }
   return 0;
 }
