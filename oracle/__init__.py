@@ -48,6 +48,7 @@ def lib() -> C.CDLL:
         _lib.e3o_block_uniform.restype = C.c_double
         _lib.e3o_inblock_uniform.restype = C.c_double
         _lib.e3o_anneal_target.restype = C.c_double
+        _lib.e3o_entropy_gap.restype = C.c_double
     return _lib
 
 
@@ -269,3 +270,17 @@ def update_temperature(s: Sched, H_t: float) -> float:
     if rc != 0:
         raise ValueError("e3o_update_temperature: invalid argument")
     return out.value
+
+
+def entropy_gap(H: float, N: int) -> float:
+    """x = beta * Delta of the two-level model that has entropy H over N entries (root x >= 1)."""
+    return float(lib().e3o_entropy_gap(C.c_double(H), C.c_int64(N)))
+
+
+def update_temperature_gap(s: Sched, H_t: float) -> float:
+    out = C.c_double()
+    rc = lib().e3o_update_temperature_gap(C.byref(s), C.c_double(H_t), C.byref(out))
+    if rc != 0:
+        raise ValueError("e3o_update_temperature_gap: invalid argument")
+    return out.value
+

@@ -34,6 +34,7 @@
  *   Algorithm 1 (Sec. 4.1)                                     -> e3o_allocate_budget
  *   Sec. 4.1 difficulty model, G_min/G_max curriculum          -> e3o_difficulty_*, e3o_budget_curriculum
  *   Eq. "tp_adj" and the annealing equation (Sec. 4.2)         -> e3o_update_temperature
+ *   Eq. "tp_relation_1" with Delta from the entropy (App. A)   -> e3o_entropy_gap, e3o_update_temperature_gap
  */
 #define _GNU_SOURCE
 #include <math.h>
@@ -571,6 +572,59 @@ int e3o_update_temperature(e3o_sched *s, double H_t, double *tau_next) {
   double lnV = log((double)s->V);
   double tau = s->tau * (1.0 + s->tau * log(alpha) / (lnV + log(lnV)));
   if (!(tau > 0.0)) return 1; /* the formula left the domain tau > 0 of App. A: state unchanged */
+  if (s->tau_max > 0.0) {
+    if (tau < s->tau_min) tau = s->tau_min;
+    if (tau > s->tau_max) tau = s->tau_max;
+  }
+  s->tau = tau;
+  s->t += 1;
+  *tau_next = tau;
+  return 0;
+}
+
+/* ------------------------------------------------------------------------- */
+/* The un-simplified scheduler of App. A.  Under the two-level model of the    */
+/* logits (one dominant logit, N-1 others at gap Delta) the entropy is          */
+/*   H ~ (N-1) beta Delta exp(-beta Delta)                                      */
+/* and scaling it by alpha needs  tau_1 ~ tau_0 (1 + tau_0 ln(alpha) / Delta)   */
+/* (Eq. "tp_relation_1").  The paper then replaces Delta by ln N + ln ln N so   */
+/* that Delta need not be estimated.  Here Delta is estimated instead, from    */
+/* the measured entropy itself by inverting the model: x = beta_0 Delta is the  */
+/* root x >= 1 of (N-1) x exp(-x) = H_t, and the update becomes                 */
+/*   tau_1 = tau_0 (1 + ln(alpha) / x).                                         */
+/* (The paper's own reduction, x = ln N + c with c = ln(ln N + c) - ln(eps), is  */
+/* this equation with N-1 ~ N; it drops -ln(eps), this function keeps it.)      */
+/* Reading: "logits can be utilized to estimate Delta" is silent on how; the    */
+/* entropy of the same logits is used.  Needs H_t <= (N-1)/e.                   */
+/* Pins: root identity; recovery of beta Delta on exact two-level rows; the     */
+/* updated temperature scales the closed-form entropy of such rows by alpha to  */
+/* within a few percent, closer than the simplified formula when Delta differs  */
+/* from ln N + ln ln N.                                                         */
+/* ------------------------------------------------------------------------- */
+double e3o_entropy_gap(double H, int64_t N) {
+  if (!(H > 0.0) || N < 3 || H > ((double)N - 1.0) / M_E) return NAN;
+  double lo = 1.0, hi = 1.0; /* x exp(-x) decreases on [1, inf): bracket the root, then bisect */
+  while (((double)N - 1.0) * hi * exp(-hi) > H) hi *= 2.0;
+  for (int it = 0; it < 200; ++it) {
+    double mid = 0.5 * (lo + hi);
+    if (((double)N - 1.0) * mid * exp(-mid) > H) lo = mid; else hi = mid;
+  }
+  return 0.5 * (lo + hi);
+}
+
+int e3o_update_temperature_gap(e3o_sched *s, double H_t, double *tau_next) {
+  if (!(H_t > 0.0) || isinf(H_t) || s->V < 3 || !(s->tau > 0.0)) return 1;
+  double x = e3o_entropy_gap(H_t, s->V);
+  if (isnan(x)) return 1;
+  if (!(s->H_init > 0.0)) {
+    s->H_init = H_t;
+    s->t += 1;
+    *tau_next = s->tau;
+    return 0;
+  }
+  double alpha = e3o_anneal_target(s) / H_t;
+  double tau = s->tau * (1.0 + log(alpha) / x);
+  if (!(tau > 0.0)) return 1;
   if (s->tau_max > 0.0) {
     if (tau < s->tau_min) tau = s->tau_min;
     if (tau > s->tau_max) tau = s->tau_max;

@@ -712,3 +712,54 @@ def test_grpo_objective_gradient_against_central_differences_and_autograd(oracle
     Jt.backward()
     assert J == pytest.approx(float(Jt), abs=1e-12)
     assert np.abs(g - x.grad.numpy()).max() < 1e-12
+
+
+# ----------------------------------------------------------------------------------------------
+# Delta-aware temperature update (Eq. tp_relation_1 with Delta estimated from the entropy, App. A)
+# ----------------------------------------------------------------------------------------------
+def _two_level_entropy(N, delta, tau):
+    b = 1.0 / tau
+    w = (N - 1) * math.exp(-b * delta)
+    return math.log(1 + w) + b * delta * w / (1 + w)      # exact entropy of one logit at +delta over N-1 at 0
+
+
+def test_entropy_gap_is_the_root_of_the_two_level_model(oracle_mod):
+    o = oracle_mod
+    for N, H in ((151936, 0.1), (151936, 2.5), (32000, 0.01), (256000, 0.7), (10, 0.5)):
+        x = o.entropy_gap(H, N)
+        assert x >= 1 and (N - 1) * x * math.exp(-x) == pytest.approx(H, rel=1e-12)
+        assert x == pytest.approx(math.log(N - 1) + math.log(x) - math.log(H), abs=1e-10)   # the paper's fixed-point form
+    assert math.isnan(o.entropy_gap(0.0, 100)) and math.isnan(o.entropy_gap(50.0, 100))
+    # on exact two-level rows of low entropy the root recovers beta * Delta
+    for delta in (16.0, 18.0, 20.0):
+        for tau in (0.8, 1.0, 1.2):
+            H = _two_level_entropy(151936, delta, tau)
+            if H < 0.5:
+                assert o.entropy_gap(H, 151936) == pytest.approx(delta / tau, rel=5e-3)
+
+
+def test_gap_update_scales_the_entropy_of_two_level_rows_by_alpha(oracle_mod):
+    o = oracle_mod
+    N = 151936
+    worse = 0
+    for delta in (16.0, 18.0, 20.0):
+        for tau in (0.8, 1.0, 1.2):
+            H0 = _two_level_entropy(N, delta, tau)
+            if H0 > 0.5:
+                continue
+            for alpha in (0.8, 1.25):
+                s = o.make_sched(tau=tau, H_init=alpha * H0, V=N)
+                t_gap = o.update_temperature_gap(s, H0)
+                s2 = o.make_sched(tau=tau, H_init=alpha * H0, V=N)
+                t_sur = o.update_temperature(s2, H0)
+                r_gap = _two_level_entropy(N, delta, t_gap) / H0
+                r_sur = _two_level_entropy(N, delta, t_sur) / H0
+                assert abs(r_gap - alpha) < 0.04, (delta, tau, alpha, r_gap)
+                assert (t_gap - tau) * (alpha - 1) > 0                  # the temperature moves the right way
+                if delta >= 18.0:      # away from Delta = ln N + ln ln N = 14.4, where the simplified formula is at home
+                    worse += abs(r_gap - alpha) > abs(r_sur - alpha)
+    assert worse == 0
+    s = o.make_sched(tau=1.0, H_init=0.3, V=N)
+    assert o.update_temperature_gap(s, 0.3) == 1.0 and s.t == 1         # alpha = 1: fixed point
+    s = o.make_sched(tau=1.0, V=N)
+    assert o.update_temperature_gap(s, 0.2) == 1.0 and s.H_init == 0.2  # first call records H_init
