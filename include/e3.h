@@ -306,6 +306,19 @@ typedef struct {
  */
 E3_API e3_status e3_update_temperature(e3_sched *s, double H_t, double *tau_next);
 
+/*
+ * The same scheduler with the logit gap Delta of App. A estimated instead of replaced by ln|V| + ln ln|V|
+ * (Eq. "tp_relation_1": tau_1 = tau_0 (1 + tau_0 ln(alpha) / Delta)), host only.  App. A models a row as one
+ * dominant logit and N-1 others at gap Delta, whose entropy is H = (N-1) x exp(-x) with x = Delta / tau_0.
+ * e3_entropy_gap returns the root x >= 1 of that equation for a measured entropy H (NaN when H <= 0, not
+ * finite, N < 3 or H > (N-1)/e, where the model has no root).  e3_update_temperature_gap then sets
+ *   tau_{t+1} = tau_t (1 + ln(alpha) / x),   alpha = H_target / H_t,
+ * with the state, first call, clamp and errors of e3_update_temperature; an H_t without a root is
+ * E3_ERR_INVALID_ARG too.
+ */
+E3_API double e3_entropy_gap(double H, int64_t N);
+E3_API e3_status e3_update_temperature_gap(e3_sched *s, double H_t, double *tau_next);
+
 /* Target entropy the scheduler holds at step s->t (H_init before annealing starts). */
 E3_API double e3_anneal_target(const e3_sched *s);
 

@@ -24,7 +24,7 @@ E3_SAMPLE_BLOCK = 256
 EXPORTS = ("e3_status_string", "e3_workspace_bytes", "e3_sample", "e3_token_logp_entropy",
            "e3_token_logp_entropy_backward", "e3_grpo_objective",
            "e3_masked_mean_entropy", "e3_masked_mean_entropy_static", "e3_group_advantage", "e3_allocate_budget", "e3_update_temperature",
-           "e3_anneal_target", "e3_difficulty_accumulate", "e3_difficulty_rank", "e3_budget_curriculum")
+           "e3_anneal_target", "e3_entropy_gap", "e3_update_temperature_gap", "e3_difficulty_accumulate", "e3_difficulty_rank", "e3_budget_curriculum")
 
 
 class E3Error(RuntimeError):
@@ -79,6 +79,10 @@ def lib() -> C.CDLL:
         L.e3_allocate_budget.argtypes = [C.c_void_p, C.c_int64, C.c_int32, C.c_int32, C.c_int32, C.c_int, C.c_void_p]
         L.e3_update_temperature.restype = C.c_int
         L.e3_update_temperature.argtypes = [C.POINTER(e3_sched), C.c_double, C.POINTER(C.c_double)]
+        L.e3_update_temperature_gap.restype = C.c_int
+        L.e3_update_temperature_gap.argtypes = [C.POINTER(e3_sched), C.c_double, C.POINTER(C.c_double)]
+        L.e3_entropy_gap.restype = C.c_double
+        L.e3_entropy_gap.argtypes = [C.c_double, C.c_int64]
         L.e3_grpo_objective.restype = C.c_int
         L.e3_grpo_objective.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_void_p, C.c_void_p,
                                         C.c_int64, C.c_float, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t,
@@ -341,6 +345,17 @@ def e3_update_temperature(s: e3_sched, H_t: float) -> float:
     st = lib().e3_update_temperature(C.byref(s), float(H_t), C.byref(out))
     _check("e3_update_temperature", st)
     return out.value
+
+
+def e3_update_temperature_gap(s: e3_sched, H_t: float) -> float:
+    out = C.c_double()
+    st = lib().e3_update_temperature_gap(C.byref(s), float(H_t), C.byref(out))
+    _check("e3_update_temperature_gap", st)
+    return out.value
+
+
+def e3_entropy_gap(H: float, N: int) -> float:
+    return lib().e3_entropy_gap(float(H), int(N))
 
 
 def e3_anneal_target(s: e3_sched) -> float:

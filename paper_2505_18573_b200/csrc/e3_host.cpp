@@ -101,6 +101,48 @@ extern "C" e3_status e3_update_temperature(e3_sched *s, double H_t, double *tau_
   return E3_OK;
 }
 
+// App. A before its last simplification: tau_1 = tau_0 (1 + tau_0 ln(alpha) / Delta), Eq. "tp_relation_1".
+// x = Delta / tau_0 is taken from the measured entropy through the two-level model H = (N-1) x exp(-x):
+// g(x) = ln((N-1)/H) + ln x - x is concave and falls for x > 1, so Newton steps started right of the root
+// come down to it monotonically and never cross it.
+extern "C" double e3_entropy_gap(double H, int64_t N) {
+  if (!(H > 0.0) || !std::isfinite(H) || N < 3) return std::nan("");
+  const double L = std::log((static_cast<double>(N) - 1.0) / H);
+  if (!(L >= 1.0)) return std::nan("");  // H above the model's maximum (N-1)/e
+  double x = 2.0 * L;                      // g(2L) = ln(2L) - L < 0: right of the root
+  for (int it = 0; it < 200; ++it) {
+    const double g = L + std::log(x) - x;
+    const double slope = 1.0 / x - 1.0;
+    if (!(slope < 0.0)) break;             // x == 1: the double root at H = (N-1)/e
+    const double next = std::max(1.0, x - g / slope);
+    if (!(next < x)) break;
+    x = next;
+  }
+  return x;
+}
+
+extern "C" e3_status e3_update_temperature_gap(e3_sched *s, double H_t, double *tau_next) {
+  if (!s || !tau_next) return E3_ERR_INVALID_ARG;
+  if (!std::isfinite(H_t) || H_t <= 0.0 || s->V < 3 || !(s->tau > 0.0) || !std::isfinite(s->tau))
+    return E3_ERR_INVALID_ARG;
+  const double x = e3_entropy_gap(H_t, s->V);
+  if (std::isnan(x)) return E3_ERR_INVALID_ARG;
+  if (!(s->H_init > 0.0)) {
+    s->H_init = H_t;
+    s->t += 1;
+    *tau_next = s->tau;
+    return E3_OK;
+  }
+  const double alpha = e3_anneal_target(s) / H_t;
+  double tau = s->tau * (1.0 + std::log(alpha) / x);
+  if (!(tau > 0.0)) return E3_ERR_INVALID_ARG;
+  if (s->tau_max > 0.0) tau = std::min(std::max(tau, s->tau_min), s->tau_max);
+  s->tau = tau;
+  s->t += 1;
+  *tau_next = tau;
+  return E3_OK;
+}
+
 // ---------------------------------------------------------------------------------------------
 // Sec. 4.1 difficulty model and the G_min / G_max curriculum
 // ---------------------------------------------------------------------------------------------

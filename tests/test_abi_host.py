@@ -120,6 +120,40 @@ def test_update_temperature_matches_oracle(e3):
     assert s.tau == 4.0 and s.t == 0
 
 
+def test_gap_based_temperature_update_matches_oracle(e3):
+    """App. A with the gap estimated from the entropy (Eq. "tp_relation_1"): root and update against the oracle."""
+    rng = np.random.default_rng(31)
+    for N in (3, 17, 32000, 151936, 256000):
+        top = (N - 1) / np.e
+        for H in list(rng.uniform(1e-6, 1.0, 20) * top) + [1e-12 * top, 1e-3, 0.3, 0.999999 * top]:
+            x = e3.e3_entropy_gap(float(H), N)
+            xo = oracle.entropy_gap(float(H), N)
+            # close to the double root at H = (N-1)/e the root is only determined to sqrt(rounding)
+            assert x == pytest.approx(xo, rel=1e-9 if H < 0.99 * top else 1e-5)
+            assert x >= 1.0
+        for bad in (0.0, -1.0, float("nan"), float("inf"), 1.001 * top):
+            assert np.isnan(e3.e3_entropy_gap(bad, N)) and np.isnan(oracle.entropy_gap(bad, N))
+    assert np.isnan(e3.e3_entropy_gap(0.1, 2))
+    for trial in range(200):
+        kw = dict(tau=float(rng.uniform(0.3, 2.0)), H_init=float(rng.uniform(0.05, 1.0)) if trial % 5 else float("nan"),
+                  t=int(rng.integers(0, 500)), t_anneal=288, t_max=480, eta=float(rng.uniform(0.5, 0.99)),
+                  V=int(rng.choice([32000, 151936, 256000])))
+        if trial % 7 == 0:
+            kw.update(tau_min=0.5, tau_max=1.5)
+        a, b = e3.make_sched(**kw), oracle.make_sched(**kw)
+        for _ in range(5):
+            H = float(rng.uniform(0.02, 1.5))
+            ta = e3.e3_update_temperature_gap(a, H)
+            tb = oracle.update_temperature_gap(b, H)
+            assert ta == pytest.approx(tb, rel=1e-10)
+            assert a.t == b.t and a.H_init == b.H_init
+    s = e3.make_sched(tau=1.0, H_init=0.2, V=1000)
+    for bad in (0.0, -1.0, float("nan"), float("inf"), 999.0):   # 999 > (N-1)/e: no root
+        with pytest.raises(e3.E3Error):
+            e3.e3_update_temperature_gap(s, bad)
+    assert s.tau == 1.0 and s.t == 0
+
+
 def test_difficulty_model_and_curriculum_match_the_oracle(oracle_mod):
     """Sec. 4.1: cumulative statistics, descending-average-reward ranks, bounds curriculum; then Algorithm 1 on the ranks."""
     import numpy as np
