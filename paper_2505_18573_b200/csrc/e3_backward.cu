@@ -6,7 +6,7 @@
 // is bound by HBM traffic (read + write).  The row's normaliser is not recomputed: the forward pass
 // returned ln p_tok, and ln p_i = (z_i - z_tok)/tau + ln p_tok.
 //
-// Work items are (row, segment of 8,192 entries); a grid of a few CTAs per SM walks them with a stride,
+// Work items are (row, segment of 8,192 entries), one CTA each,
 // each thread moving 16-byte vectors (8 bf16 or 4 fp32 logits) with streaming loads and stores.
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
@@ -199,10 +199,9 @@ extern "C" e3_status e3_token_logp_entropy_backward(const void *logits, e3_dtype
   p.logp = logp; p.ent = ent; p.g_logp = g_logp; p.g_ent = g_ent;
   p.segs_per_row = (V + kSegE - 1) / kSegE;
   p.items = rows * p.segs_per_row;
-  int dev = 0, sms = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
-    return E3_ERR_CUDA;
-  const int64_t cap = (int64_t)sms * 8;
+  // One CTA per item (measured faster than a grid of a few CTAs per SM that loops: the hardware hands
+  // out CTAs as SMs become free, which evens out the tail); the loop only matters beyond 2^31 - 1 items.
+  const int64_t cap = 0x7fffffff;
   const unsigned grid = (unsigned)(p.items < cap ? p.items : cap);
   const bool aligned = !misaligned(logits, 16) && !misaligned(dlogits, 16) && (row_stride * esize) % 16 == 0 &&
                        (dlogits_stride * esize) % 16 == 0;

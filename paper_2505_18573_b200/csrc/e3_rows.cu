@@ -1094,7 +1094,7 @@ __device__ __forceinline__ const char *row_ptr(const RowsParams &p, int64_t row)
 // Row epilogue (one thread, fp64).  zt: logit of the token whose log-probability is wanted.
 // ---------------------------------------------------------------------------------------------
 __device__ __forceinline__ void finish_row(const RowsParams &p, int64_t row, const RowInfo &ri, float Mf, float Zf,
-                                           float Wf, int idx, int err, bool have_zt, float zt) {
+                                           float Wf, int idx, int err, bool have_zt, float zt, bool store) {
   const double M = Mf, Z = Zf, W = Wf;
   const bool sample = p.mode == kModeSample;
   int tok = -1;
@@ -1107,6 +1107,7 @@ __device__ __forceinline__ void finish_row(const RowsParams &p, int64_t row, con
     if (sample) tok = idx;
     if (have_zt) logp = (float)(((double)zt * (double)ri.c - M) * kLn2 - lnZ);
   }
+  if (!store) return;
   if (sample) p.out_tok[row] = tok;
   if (p.out_logp) p.out_logp[row] = logp;
   if (p.out_ent) p.out_ent[row] = ent;
@@ -1205,8 +1206,10 @@ __device__ __noinline__ int draw_in_block_exact(const EvalCtx &x, int b, int lan
   return tok;
 }
 
-// The same draw in fp32.  When the threshold comes closer than 1e-4 of the block sum to a prefix
-// boundary (fp32 prefix sums are good to about 1e-5) the exact form decides.  z_tok: logit of the token.
+// The same draw in fp32.  The prefix sums are good to about 3e-6 of the block sum (entries that matter
+// have |t| < 25, so the rounding of t costs 2e-6 relative, `ex2` 2e-7, the 13 additions 8e-7); when the
+// threshold comes closer than ten times that to a prefix boundary the exact form decides.
+// z_tok: logit of the token.
 template <int DT>
 __device__ __noinline__ int draw_in_block(const EvalCtx &x, int b, int lane, float &z_tok) {
   float z[8];
@@ -1251,7 +1254,7 @@ __device__ __noinline__ int draw_in_block(const EvalCtx &x, int b, int lane, flo
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) gap = fminf(gap, __shfl_xor_sync(0xffffffffu, gap, o));
     const uint32_t found = __ballot_sync(0xffffffffu, hit >= 0);
-    exact = !(gap > 1e-4f * total) || found == 0u || !(total > 0.f) || !(total < CUDART_INF_F);
+    exact = !(gap > 3e-5f * total) || found == 0u || !(total > 0.f) || !(total < CUDART_INF_F);
     if (!exact) {
       const int src = __ffs(found) - 1;
       const int k = __shfl_sync(0xffffffffu, hit, src);
@@ -1677,9 +1680,22 @@ __global__ void __launch_bounds__(kThreads, 2) rows_kernel(const __grid_constant
     u64 *const pieces = reinterpret_cast<u64 *>(p.ws_pieces);
     constexpr int kPieceStride = (int)(kPieceBytes / 8);
     const bool sample = p.mode == kModeSample;
-    while (it.next(p, s, ri)) {
+    // The code below runs once or twice per CTA, the last time at the very end of the CTA's life, when
+    // nothing hides it, and a first run through cold code is dominated by instruction fetches (several
+    // times the warm time).  So the warp rehearses it while the consumers work on the first piece: pass
+    // number p.rehearse takes the first piece's descriptors and made-up sums through the same
+    // instructions with every store, barrier operation and workspace write switched off.  (The pass number
+    // is a kernel argument so that the compiler keeps a single copy of the loop body.)
+    for (int pass = 0;; ++pass) {
+      const bool ghost = pass == p.rehearse;
+      if (ghost) {
+        SegIter peek = it;
+        if (!peek.next(p, s, ri)) continue;
+      } else if (!it.next(p, s, ri)) {
+        break;
+      }
       if (ri.masked || ri.invalid) {
-        if (s.starts && lane == 0) write_skipped(p, s.row, ri);
+        if (!ghost && s.starts && lane == 0) write_skipped(p, s.row, ri);
         continue;
       }
       // the target's logit is fetched while the consumers work on the piece
@@ -1690,12 +1706,12 @@ __global__ void __launch_bounds__(kThreads, 2) rows_kernel(const __grid_constant
         if (target >= 0 && target < p.V) zt = load_elem<DT>(row_ptr<DT>(p, s.row), target);
       }
       const uint32_t slot = n % kSlots, use = n / kSlots;
-      mbar_wait_warp(&sm.wfull[slot], use & 1u, sm, lane);
+      if (!ghost) mbar_wait_warp(&sm.wfull[slot], use & 1u, sm, lane);
       Piece pc;
       pc.M = 0.f; pc.Z = 0.f; pc.W = 0.f; pc.zf = 0.f; pc.err = 0; pc.pad = 0;
       Top3 top;
       top3_reset(top);
-      if (lane < kStreamWarps) {
+      if (!ghost && lane < kStreamWarps) {
         const WarpPartial &w = sm.wpart[slot][lane];
         pc.M = w.M; pc.Z = w.Z; pc.W = w.W; pc.err = w.err; pc.zf = w.zf;
         if (SAMPLER >= 0) {
@@ -1704,19 +1720,21 @@ __global__ void __launch_bounds__(kThreads, 2) rows_kernel(const __grid_constant
         }
       }
       __syncwarp();
-      if (lane == 0) mbar_arrive(&sm.wfree[slot]);
-      ++n;
+      if (!ghost) {
+        if (lane == 0) mbar_arrive(&sm.wfree[slot]);
+        ++n;
+      }
       // The order of every merge below is fixed by lane and piece numbers alone, so the result does not
       // depend on which CTA ends up finishing the row.
       warp_merge(pc, top, SAMPLER >= 0);
       if (*reinterpret_cast<volatile int *>(&sm.timeout)) pc.err |= kErrTimeout;
       bool fin = s.whole;
-      if (!s.whole) {
+      if (!s.whole || (ghost && pieces != nullptr)) {
         // A piece of a cut row.  Store it, then (after a sequentially consistent fence) look for the
         // row's other pieces: of all CTAs that hold a piece, the one whose fence comes last is sure to
         // find them all and finishes the row.  Two CTAs may both find all pieces; they then write the
         // same values.  Nobody waits for anybody.
-        if (lane == 0) {
+        if (lane == 0 && !ghost) {
 #pragma unroll
           for (int i = 0; i < 3; ++i) { pc.ty[i] = top.y[i]; pc.tb[i] = top.b[i]; }
           piece_store(pieces + ((size_t)blockIdx.x * 2 + (s.first ? 0 : 1)) * kPieceStride, p.call_id, pc);
@@ -1743,7 +1761,13 @@ __global__ void __launch_bounds__(kThreads, 2) rows_kernel(const __grid_constant
           }
         }
         fin = __all_sync(0xffffffffu, ok);
-        if (fin) warp_merge(pc, top, SAMPLER >= 0);
+        if (fin || ghost) warp_merge(pc, top, SAMPLER >= 0);
+      }
+      if (ghost) {  // made-up sums and a leader that exists in every row: entry 0 / block 0
+        fin = true;
+        pc.M = 0.f; pc.Z = 1.f; pc.W = 0.f; pc.zf = 0.f; pc.err = 0;
+        top3_reset(top);
+        top.y[0] = 0.f; top.b[0] = 0;
       }
       if (!fin) continue;
       int id = -1;
@@ -1767,7 +1791,7 @@ __global__ void __launch_bounds__(kThreads, 2) rows_kernel(const __grid_constant
           have_zt = id >= 0;
         }
       }
-      if (lane == 0) finish_row(p, s.row, ri, pc.M, pc.Z, pc.W, id, pc.err, have_zt, zt);
+      if (lane == 0) finish_row(p, s.row, ri, pc.M, pc.Z, pc.W, id, pc.err, have_zt, zt, !ghost);
     }
   }
 }
@@ -1837,6 +1861,7 @@ cudaError_t launch_one(RowsParams p, void *workspace, size_t workspace_bytes, cu
   p.tiles_r = tiles % grid;
   p.ws_pieces = can_cut ? static_cast<unsigned char *>(workspace) : nullptr;
   p.call_id = next_call_id();
+  p.rehearse = 0;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)grid);
   cfg.blockDim = dim3(kThreads);

@@ -43,6 +43,7 @@ struct RowsParams {
   // cut rows: partial states in the caller's workspace
   unsigned char *ws_pieces;          // [grid][2] pieces of kPieceBytes, every word tagged with the call id
   unsigned long long call_id;        // unique per call within the process (48 bits)
+  int rehearse;                      // pass of the finishing warp that is a dry run (0), -1: none
 };
 
 size_t rows_workspace_bytes();
