@@ -647,13 +647,12 @@ __device__ __forceinline__ void top3_insert(Top3 &t, float y, int b) {
 
 struct BlockState {
   Top3 top;
-  float S, ref;  // parked block: sum 2^(z c + ref)
-  int b;         // its block index
-  int it;        // steps taken in this segment (warp-uniform)
+  float ref;  // parked block: its lane sums were taken under this reference
+  int b;      // its block index, -1: none
 };
 __device__ __forceinline__ void block_state_reset(BlockState &bs) {
   top3_reset(bs.top);
-  bs.S = 0.f; bs.ref = 0.f; bs.b = -1; bs.it = 0;
+  bs.ref = 0.f; bs.b = -1;
 }
 
 // fp32 Gumbel variate of block b: u = (x + 1/2) 2^-32, g = -ln(-ln u)
@@ -671,36 +670,48 @@ __device__ __forceinline__ float block_gumbel_f32(const uint32_t *rk, uint32_t g
   return -lg2f(a) * kLn2f;
 }
 
-__device__ __noinline__ void block_flush(const uint32_t *rk, uint32_t grow, uint32_t ctr_lo, uint32_t ctr_hi8,
-                                         BlockState &bs) {
-  if (bs.b >= 0 && bs.S > 0.f) {
-    const float L = (lg2f(bs.S) - bs.ref) * kLn2f;  // ln sum_i exp(s_i) over the block
-    top3_insert(bs.top, L + block_gumbel_f32(rk, grow, ctr_lo, ctr_hi8, bs.b), bs.b);
+// fp32 score of a block: ln sum_i exp(s_i) + g_b, from S = sum 2^(z c + ref).  Out of line (scalars in,
+// scalar out) so that the streaming loop stays short and its state stays in registers.
+__device__ __noinline__ float block_score(const uint32_t *rk, uint32_t grow, uint32_t ctr_lo, uint32_t ctr_hi8, float S,
+                                          float ref, int b) {
+  return (lg2f(S) - ref) * kLn2f + block_gumbel_f32(rk, grow, ctr_lo, ctr_hi8, b);
+}
+
+// Adds up the parked blocks of the warp (lane j of each group of kLB lanes owns the block of step j of
+// the current round; its lane sums sit in the warp's scratch) and enters their scores in the lane's list.
+template <int DT>
+__device__ __forceinline__ void block_flush(const uint32_t *rk, uint32_t grow, uint32_t ctr_lo, uint32_t ctr_hi8,
+                                            BlockState &bs, const float *scratch, int lane) {
+  constexpr int kLB = Fmt<DT>::kLB;
+  __syncwarp();
+  const float4 *src = reinterpret_cast<const float4 *>(scratch + (lane & (kLB - 1)) * 32 + (lane & ~(kLB - 1)));
+  float S = 0.f;
+#pragma unroll
+  for (int i = 0; i < kLB / 4; ++i) {
+    const float4 v = src[i];
+    S += (v.x + v.y) + (v.z + v.w);
   }
-  bs.S = 0.f;
+  __syncwarp();  // the scratch is written again in the next step
+  if (bs.b >= 0 && S > 0.f) top3_insert(bs.top, block_score(rk, grow, ctr_lo, ctr_hi8, S, bs.ref, bs.b), bs.b);
   bs.b = -1;
 }
 
-// One step of a warp: every lane brings the sum of 2^t over its entries of this step (all lanes under
-// the reference nRc), which lie in block `b`.
+// Step `it` of a warp in its row piece: every lane brings the sum of 2^t over its entries of this step
+// (all lanes under the reference nRc), which lie in block `b`; kLB neighbouring lanes share a block.
+// The lane sums go to the warp's scratch in shared memory and are added up only every kLB steps: one
+// read instead of a chain of shuffles at the end of every step.
 template <int DT>
 __device__ __forceinline__ void block_step(float zlane, int b, float nRc, const uint32_t *rk, uint32_t grow,
-                                           uint32_t ctr_lo, uint32_t ctr_hi8, BlockState &bs, int lane) {
+                                           uint32_t ctr_lo, uint32_t ctr_hi8, BlockState &bs, float *scratch,
+                                           int lane, int it) {
   constexpr int kLB = Fmt<DT>::kLB;
-  float sb = zlane;
-#pragma unroll
-  for (int o = 1; o < kLB; o <<= 1) sb += __shfl_xor_sync(0xffffffffu, sb, o);
-  if ((bs.it & (kLB - 1)) == (lane & (kLB - 1))) {
-    bs.S = sb;
+  const int j = it & (kLB - 1);
+  scratch[j * 32 + lane] = zlane;
+  if (j == (lane & (kLB - 1))) {
     bs.ref = nRc;
     bs.b = b;
   }
-  ++bs.it;
-  if ((bs.it & (kLB - 1)) == 0) {
-    BlockState t = bs;
-    block_flush(rk, grow, ctr_lo, ctr_hi8, t);
-    bs = t;
-  }
+  if (j == kLB - 1) block_flush<DT>(rk, grow, ctr_lo, ctr_hi8, bs, scratch, lane);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -1354,7 +1365,7 @@ __device__ __noinline__ int settle_exact(const EvalCtx &x, const Top3 &top, floa
 // ---------------------------------------------------------------------------------------------
 template <int DT, int SAMPLER, bool RING>
 __global__ void __launch_bounds__(kThreads, 2) rows_kernel(const __grid_constant__ RowsParams p) {
-  extern __shared__ __align__(128) unsigned char dyn[];  // ring, then the candidate queues of sampler 0
+  extern __shared__ __align__(128) unsigned char dyn[];  // ring, then sampler 0: candidate queues, sampler 1: lane sums
   __shared__ Smem sm;
   using F = Fmt<DT>;
   constexpr int kEsize = F::kEsize;
@@ -1391,6 +1402,8 @@ __global__ void __launch_bounds__(kThreads, 2) rows_kernel(const __grid_constant
     uint32_t n = 0;                 // segments handed to the finishing warp so far
     const uint32_t *const rk = p.round_key;
     unsigned char *const queue = dyn + (RING ? kStages * kStageBytes : 0) + warp * F::kQueueBytes;
+    // sampler 1: the warp's lane sums of the last kLB steps
+    float *const bscratch = reinterpret_cast<float *>(dyn + (RING ? kStages * kStageBytes : 0)) + warp * (F::kLB * 32);
     // vector order of this lane inside its 64 bytes (the lanes of a quarter warp hit distinct banks)
     const int rot = (lane >> 1) & 3;
     while (it.next(p, s, ri)) {
@@ -1446,10 +1459,10 @@ __global__ void __launch_bounds__(kThreads, 2) rows_kernel(const __grid_constant
           const int lim = fast_end < cs + kChunkE ? fast_end : cs + kChunkE;
           if (c == 0) {
             SeedIO sd;
-            sd.best = best;
+            if (SAMPLER == 0) sd.best = best;
             E3_MAKE_CTX(ex);
             seed_piece<DT, SAMPLER>(sd, ex, lane_data, e_lane, lim, sm);
-            best = sd.best;
+            if (SAMPLER == 0) best = sd.best;
             if (sd.R0 > -CUDART_INF_F) {
               const float nRc = -sd.R0 * ri.c;
               if (fabsf(nRc) < CUDART_INF_F) { acc.R = sd.R0; acc.nRc = nRc; }
@@ -1469,10 +1482,12 @@ __global__ void __launch_bounds__(kThreads, 2) rows_kernel(const __grid_constant
             const int owner = (fast_end - cs) / kLaneE;  // thread whose 64 bytes would hold it
             if ((owner >> 5) == warp) {
               SlowIO io;
-              io.acc = acc; io.best = best; io.err = err; io.zsum = 0.f;
+              io.acc = acc; io.err = err; io.zsum = 0.f;
+              if (SAMPLER == 0) io.best = best;
               E3_MAKE_CTX(ex);
               slow_groups<DT, SAMPLER, true>(io, ex, owner == tid ? fast_end : s.e_hi, s.e_hi, ri.c, sm);
-              acc = io.acc; best = io.best; err = io.err;
+              acc = io.acc; err = io.err;
+              if (SAMPLER == 0) best = io.best;
               zextra = io.zsum;
               if (SAMPLER == 0) ethr = gate_threshold(best.enc, acc.nRc);
             }
@@ -1561,21 +1576,33 @@ __global__ void __launch_bounds__(kThreads, 2) rows_kernel(const __grid_constant
               }
             }
           }
-          if (SAMPLER == 1) block_step<DT>(zl, e_lane >> 8, acc.nRc, rk, grow, p.ctr_lo, p.ctr_hi8, bs, lane);
+          if (SAMPLER == 1) block_step<DT>(zl, e_lane >> 8, acc.nRc, rk, grow, p.ctr_lo, p.ctr_hi8, bs, bscratch, lane, c);
         } else if (ri.greedy) {
           SlowIO io;
-          io.acc = acc; io.best = best; io.err = err; io.zsum = 0.f;
+          io.acc = acc; io.err = err; io.zsum = 0.f;
+          if (SAMPLER != 0) {  // the running maximum lives in the list of blocks, which greedy rows do not use
+            io.best.y[0] = bs.top.y[0]; io.best.b[0] = bs.top.b[0];
+          } else {
+            io.best = best;
+          }
           greedy_groups<DT>(io, row, RING ? stage_ptr + tid * kLaneBytes : nullptr, e_lane,
                             fast_end < cs + kChunkE ? fast_end : cs + kChunkE, s.e_hi);
-          best = io.best; err = io.err;
+          err = io.err;
+          if (SAMPLER != 0) {
+            bs.top.y[0] = io.best.y[0]; bs.top.b[0] = io.best.b[0];
+          } else {
+            best = io.best;
+          }
         } else {
           // rows that cannot use the ring: everything through the guarded form
           SlowIO io;
-          io.acc = acc; io.best = best; io.err = err; io.zsum = 0.f;
+          io.acc = acc; io.err = err; io.zsum = 0.f;
+          if (SAMPLER == 0) io.best = best;
           E3_MAKE_CTX(ex);
           slow_groups<DT, SAMPLER, true>(io, ex, e_lane < s.e_hi ? e_lane : s.e_hi, s.e_hi, ri.c, sm);
-          acc = io.acc; best = io.best; err = io.err;
-          if (SAMPLER == 1) block_step<DT>(io.zsum, e_lane >> 8, acc.nRc, rk, grow, p.ctr_lo, p.ctr_hi8, bs, lane);
+          acc = io.acc; err = io.err;
+          if (SAMPLER == 0) best = io.best;
+          if (SAMPLER == 1) block_step<DT>(io.zsum, e_lane >> 8, acc.nRc, rk, grow, p.ctr_lo, p.ctr_hi8, bs, bscratch, lane, c);
         }
         if (RING) {
           __syncwarp();
@@ -1590,9 +1617,8 @@ __global__ void __launch_bounds__(kThreads, 2) rows_kernel(const __grid_constant
         qn = 0;
       }
       if (SAMPLER == 1 && !ri.greedy) {
-        BlockState t = bs;
-        block_flush(rk, grow, p.ctr_lo, p.ctr_hi8, t);
-        bs = t;
+        // blocks of the unfinished round: lanes whose step has not come hold no block (b = -1)
+        block_flush<DT>(rk, grow, p.ctr_lo, p.ctr_hi8, bs, bscratch, lane);
       }
 
       AccS fin = to_scalar(acc);
@@ -1618,8 +1644,8 @@ __global__ void __launch_bounds__(kThreads, 2) rows_kernel(const __grid_constant
       Piece pw;
       pw.M = -fin.nRc; pw.Z = fin.Z; pw.W = fin.W;
       if (fin.R == -CUDART_INF_F) { pw.M = 0.f; pw.Z = 0.f; pw.W = 0.f; }
-      pw.zf = best.zf; pw.err = err;
-      if (SAMPLER != 1 || ri.greedy) {  // sampler 0 and greedy rows: the thread's leaders; sampler 1: its blocks
+      pw.zf = SAMPLER == 0 ? best.zf : 0.f; pw.err = err;
+      if (SAMPLER == 0) {  // the thread's leaders; sampler 1 has its blocks there (greedy rows: the maximum) already
 #pragma unroll
         for (int i = 0; i < 3; ++i) { bs.top.y[i] = best.y[i]; bs.top.b[i] = best.b[i]; }
       }
@@ -1806,7 +1832,8 @@ struct KernelSetup {
 
 template <int DT, int SAMPLER, bool RING>
 constexpr size_t dyn_smem_bytes() {
-  return (RING ? (size_t)kStages * kStageBytes : 0) + (SAMPLER == 0 ? (size_t)kStreamWarps * Fmt<DT>::kQueueBytes : 0);
+  return (RING ? (size_t)kStages * kStageBytes : 0) + (SAMPLER == 0 ? (size_t)kStreamWarps * Fmt<DT>::kQueueBytes : 0) +
+         (SAMPLER == 1 ? (size_t)kStreamWarps * Fmt<DT>::kLB * 32 * sizeof(float) : 0);
 }
 
 template <int DT, int SAMPLER, bool RING>
