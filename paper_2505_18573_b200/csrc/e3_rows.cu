@@ -148,7 +148,7 @@ struct Seg {
 // Running sums of a consumer thread, two fp32 lanes per register pair.
 struct Acc {
   float R, nRc;      // reference logit and -R*c; R = -inf, nRc = kNoRef: no reference yet
-  f2 Z2, Wa2, Wb2;   // Z = sum of both halves of Z2, W = sum of the four halves of Wa2, Wb2
+  f2 Z2, W2;         // Z = sum of both halves of Z2, W likewise
 };
 // The same state as plain scalars (careful form).
 struct AccS {
@@ -352,22 +352,21 @@ constexpr float kNoRef = 1e30f;  // nRc of a state without reference: the first 
 __device__ __forceinline__ void acc_reset(Acc &a) {
   a.R = -CUDART_INF_F;
   a.nRc = kNoRef;
-  a.Z2 = a.Wa2 = a.Wb2 = pack2f(0.f, 0.f);
+  a.Z2 = a.W2 = pack2f(0.f, 0.f);
 }
 __device__ __forceinline__ AccS to_scalar(const Acc &a) {
   AccS s;
   s.R = a.R;
   s.nRc = a.nRc;
   s.Z = sum2(a.Z2);
-  s.W = sum2(a.Wa2) + sum2(a.Wb2);
+  s.W = sum2(a.W2);
   return s;
 }
 __device__ __forceinline__ void from_scalar(Acc &a, const AccS &s) {
   a.R = s.R;
   a.nRc = s.nRc;
   a.Z2 = pack2f(s.Z, 0.f);
-  a.Wa2 = pack2f(s.W, 0.f);
-  a.Wb2 = pack2f(0.f, 0.f);
+  a.W2 = pack2f(s.W, 0.f);
 }
 
 // Careful form for one group: accepts any values.  -inf entries carry no weight, NaN and +inf flag the
@@ -436,11 +435,11 @@ __device__ __forceinline__ float group_max(const uint4 *v) {
   }
 }
 
-// Streaming form for one group held in raw 16-byte vectors (any order): adds sum 2^t t to (Wa2, Wb2),
+// Streaming form for one group held in raw 16-byte vectors (any order): returns the packed sum of 2^t t in Wg2,
 // returns the packed group sum of 2^t in Zg2 and its scalar value.
 template <int DT>
-__device__ __forceinline__ float hot_group(const uint4 *v, f2 c2, f2 nRc2, f2 &Wa2, f2 &Wb2, f2 &Zg2) {
-  f2 Za = pack2f(0.f, 0.f), Zb = pack2f(0.f, 0.f);
+__device__ __forceinline__ float hot_group(const uint4 *v, f2 c2, f2 nRc2, f2 &Wg2, f2 &Zg2) {
+  f2 Za = pack2f(0.f, 0.f), Zb = pack2f(0.f, 0.f), Wa2 = pack2f(0.f, 0.f), Wb2 = pack2f(0.f, 0.f);
 #pragma unroll
   for (int q = 0; q < Fmt<DT>::kVG; ++q) {
     const uint32_t w[4] = {v[q].x, v[q].y, v[q].z, v[q].w};
@@ -465,6 +464,7 @@ __device__ __forceinline__ float hot_group(const uint4 *v, f2 c2, f2 nRc2, f2 &W
     }
   }
   Zg2 = add2(Za, Zb);
+  Wg2 = add2(Wa2, Wb2);
   return sum2(Zg2);
 }
 
@@ -1510,14 +1510,12 @@ __global__ void __launch_bounds__(kThreads, 2) rows_kernel(const __grid_constant
               for (int i = 0; i < kVG; ++i) raw[i] = pv[(i ^ rot) & (kVG - 1)];
             }
             float Zg = 0.f;
-            f2 Zg2 = pack2f(0.f, 0.f);
-            f2 Wa_in = acc.Wa2, Wb_in = acc.Wb2;
+            f2 Zg2 = pack2f(0.f, 0.f), Wg2 = pack2f(0.f, 0.f);  // the group's sums; they join the state once they are known to be sound
 #pragma unroll 1
             for (int attempt = 0;; ++attempt) {
-              if (have) Zg = hot_group<DT>(raw, pack2f(ri.c, ri.c), pack2f(acc.nRc, acc.nRc), acc.Wa2, acc.Wb2, Zg2);
+              if (have) Zg = hot_group<DT>(raw, pack2f(ri.c, ri.c), pack2f(acc.nRc, acc.nRc), Wg2, Zg2);
               if (!__any_sync(0xffffffffu, have && !(Zg <= kGroupSumMax))) break;
               // the reference is stale for some lane (or a value is not finite)
-              acc.Wa2 = Wa_in; acc.Wb2 = Wb_in;
               const float gm = have ? group_max<DT>(raw) : -CUDART_INF_F;
               const float newR = dec_float(__reduce_max_sync(0xffffffffu, enc_float(gm)));
               const float nRc = -newR * ri.c;
@@ -1526,13 +1524,11 @@ __global__ void __launch_bounds__(kThreads, 2) rows_kernel(const __grid_constant
                 const float d = nRc - acc.nRc;
                 const float f = acc.R == -CUDART_INF_F ? 0.f : ex2f(d);
                 const f2 ff = pack2f(f, f);
-                acc.Wa2 = mul2(ff, fma2(pack2f(d, d), acc.Z2, acc.Wa2));
-                acc.Wb2 = mul2(ff, acc.Wb2);
+                acc.W2 = mul2(ff, fma2(pack2f(d, d), acc.Z2, acc.W2));
                 acc.Z2 = mul2(ff, acc.Z2);
-                if (f == 0.f) acc.Z2 = acc.Wa2 = acc.Wb2 = pack2f(0.f, 0.f);
+                if (f == 0.f) acc.Z2 = acc.W2 = pack2f(0.f, 0.f);
                 acc.R = newR; acc.nRc = nRc;
                 zl *= f;
-                Wa_in = acc.Wa2; Wb_in = acc.Wb2;
                 if (SAMPLER == 0) ethr = gate_threshold(best.enc, acc.nRc);
                 continue;
               }
@@ -1543,11 +1539,12 @@ __global__ void __launch_bounds__(kThreads, 2) rows_kernel(const __grid_constant
               redo_step<DT, true>(io, lane_data, have ? (1 << gn) : 0, ri.c);
               acc = io.acc; err = io.err; zl = io.Zextra;
               Zg = io.Zg[gn];
-              Zg2 = pack2f(0.f, 0.f);  // the careful form has added the group already
+              Zg2 = Wg2 = pack2f(0.f, 0.f);  // the careful form has added the group already
               if (SAMPLER == 0) ethr = gate_threshold(best.enc, acc.nRc);
               break;
             }
             acc.Z2 = add2(acc.Z2, Zg2);
+            acc.W2 = add2(acc.W2, Wg2);
             zl += Zg;
             if (SAMPLER == 0) {
               const uint4 cb = philox(rk, (uint32_t)g0 >> 4, grow, p.ctr_lo, p.ctr_hi8 | 0u);
