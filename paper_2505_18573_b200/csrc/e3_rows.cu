@@ -437,11 +437,11 @@ __device__ __forceinline__ float group_max(const uint4 *v) {
 
 // Streaming form for one group held in raw 16-byte vectors (any order): returns the packed sum of 2^t t in Wg2,
 // returns the packed group sum of 2^t in Zg2 and its scalar value.
-template <int DT>
-__device__ __forceinline__ float hot_group(const uint4 *v, f2 c2, f2 nRc2, f2 &Wg2, f2 &Zg2) {
+template <int DT, int NV>
+__device__ __forceinline__ float hot_vectors(const uint4 *v, f2 c2, f2 nRc2, f2 &Wg2, f2 &Zg2) {
   f2 Za = pack2f(0.f, 0.f), Zb = pack2f(0.f, 0.f), Wa2 = pack2f(0.f, 0.f), Wb2 = pack2f(0.f, 0.f);
 #pragma unroll
-  for (int q = 0; q < Fmt<DT>::kVG; ++q) {
+  for (int q = 0; q < NV; ++q) {
     const uint32_t w[4] = {v[q].x, v[q].y, v[q].z, v[q].w};
 #pragma unroll
     for (int j = 0; j < (DT == 1 ? 4 : 2); ++j) {
@@ -466,6 +466,11 @@ __device__ __forceinline__ float hot_group(const uint4 *v, f2 c2, f2 nRc2, f2 &W
   Zg2 = add2(Za, Zb);
   Wg2 = add2(Wa2, Wb2);
   return sum2(Zg2);
+}
+
+template <int DT>
+__device__ __forceinline__ float hot_group(const uint4 *v, f2 c2, f2 nRc2, f2 &Wg2, f2 &Zg2) {
+  return hot_vectors<DT, Fmt<DT>::kVG>(v, c2, nRc2, Wg2, Zg2);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -1498,8 +1503,27 @@ __global__ void __launch_bounds__(kThreads, 2) rows_kernel(const __grid_constant
           // distinct banks.  All lanes of the warp share one reference logit.
           const int ga = kG == 2 ? (rot >> 1) : 0;
           float zl = zextra;  // sampler 1: this thread's share of its block
+          // Without the per-group work of sampler 0, a stage that lies wholly inside the row is taken in
+          // one piece: the thread's 64 bytes in straight-line code and one check for the warp.  If the
+          // check fails (stale reference, a value that is not finite) nothing has been added yet and
+          // the turns below deal with the stage.
+          bool stage_done = false;
+          if (SAMPLER != 0 && fast_end >= cs + kChunkE) {
+            uint4 raw[4];
+            const uint4 *pv = reinterpret_cast<const uint4 *>(lane_data);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) raw[i] = pv[i ^ rot];
+            f2 Zs2, Ws2;
+            const float Zs = hot_vectors<DT, 4>(raw, pack2f(ri.c, ri.c), pack2f(acc.nRc, acc.nRc), Ws2, Zs2);
+            if (!__any_sync(0xffffffffu, !(Zs <= kGroupSumMax))) {
+              acc.Z2 = add2(acc.Z2, Zs2);
+              acc.W2 = add2(acc.W2, Ws2);
+              zl += Zs;
+              stage_done = true;
+            }
+          }
 #pragma unroll 1
-          for (int gi = 0; gi < kG; ++gi) {
+          for (int gi = stage_done ? kG : 0; gi < kG; ++gi) {
             const int gn = gi ^ ga;
             const int g0 = e_lane + (gn << 4);
             const bool have = g0 + kGroup <= lim;
