@@ -689,11 +689,12 @@ __device__ __forceinline__ void block_flush(const uint32_t *rk, uint32_t grow, u
                                             BlockState &bs, const float *scratch, int lane) {
   constexpr int kLB = Fmt<DT>::kLB;
   __syncwarp();
-  const float4 *src = reinterpret_cast<const float4 *>(scratch + (lane & (kLB - 1)) * 32 + (lane & ~(kLB - 1)));
+  // row j of the scratch is rotated by 8 j columns, which spreads the lanes' reads over the banks
+  const int j = lane & (kLB - 1), col0 = (lane & ~(kLB - 1)) + 8 * j;
   float S = 0.f;
 #pragma unroll
   for (int i = 0; i < kLB / 4; ++i) {
-    const float4 v = src[i];
+    const float4 v = *reinterpret_cast<const float4 *>(scratch + j * 32 + ((col0 + 4 * i) & 31));
     S += (v.x + v.y) + (v.z + v.w);
   }
   __syncwarp();  // the scratch is written again in the next step
@@ -711,7 +712,7 @@ __device__ __forceinline__ void block_step(float zlane, int b, float nRc, const 
                                            int lane, int it) {
   constexpr int kLB = Fmt<DT>::kLB;
   const int j = it & (kLB - 1);
-  scratch[j * 32 + lane] = zlane;
+  scratch[j * 32 + ((lane + 8 * j) & 31)] = zlane;
   if (j == (lane & (kLB - 1))) {
     bs.ref = nRc;
     bs.b = b;
