@@ -847,6 +847,21 @@ __device__ __noinline__ void greedy_groups(SlowIO &io, const char *row, const un
   }
 }
 
+// The reference part of seed_piece alone, in line (no per-entry work): the largest finite logit among the
+// first groups of the warp's lanes, -inf if there is none.
+template <int DT>
+__device__ __forceinline__ float seed_reference(const unsigned char *lane_data, int e_lane, int lim) {
+  float gmax = -CUDART_INF_F;
+  if (e_lane + kGroup <= lim) {
+    uint4 v[Fmt<DT>::kVG];
+#pragma unroll
+    for (int i = 0; i < Fmt<DT>::kVG; ++i) v[i] = reinterpret_cast<const uint4 *>(lane_data)[i];
+    gmax = group_max<DT>(v);
+  }
+  if (!(gmax < CUDART_INF_F)) gmax = -CUDART_INF_F;
+  return dec_float(__reduce_max_sync(0xffffffffu, enc_float(gmax)));
+}
+
 struct SeedIO {
   float R0;  // warp-wide reference, -inf = none found
   Best best;
@@ -1050,8 +1065,17 @@ struct Walker {
     }
     const int64_t len = run_length(p);
     if (rel >= len) return false;
-    const int64_t t = first_tile_of(p, blockIdx.x) + rel;
-    const int64_t row = quot(p, t, p.tiles_per_row), tin = t - row * p.tiles_per_row;
+    // only the CTA's first piece can start inside a row: every later one starts the row after `s.row`
+    // (s still holds the piece handed out before)
+    int64_t row, tin;
+    if (rel == 0) {
+      const int64_t t = first_tile_of(p, blockIdx.x);
+      row = quot(p, t, p.tiles_per_row);
+      tin = t - row * p.tiles_per_row;
+    } else {
+      row = s.row + 1;
+      tin = 0;
+    }
     const int64_t n = p.tiles_per_row - tin < len - rel ? p.tiles_per_row - tin : len - rel;
     const int64_t lo = tin * kTile, hi = (tin + n) * kTile;
     s.row = row;
@@ -1464,14 +1488,20 @@ __global__ void __launch_bounds__(kThreads, 2) rows_kernel(const __grid_constant
           const unsigned char *lane_data = stage_ptr + tid * kLaneBytes;
           const int lim = fast_end < cs + kChunkE ? fast_end : cs + kChunkE;
           if (c == 0) {
-            SeedIO sd;
-            if (SAMPLER == 0) sd.best = best;
-            E3_MAKE_CTX(ex);
-            seed_piece<DT, SAMPLER>(sd, ex, lane_data, e_lane, lim, sm);
-            if (SAMPLER == 0) best = sd.best;
-            if (sd.R0 > -CUDART_INF_F) {
-              const float nRc = -sd.R0 * ri.c;
-              if (fabsf(nRc) < CUDART_INF_F) { acc.R = sd.R0; acc.nRc = nRc; }
+            float R0;
+            if (SAMPLER == 0) {
+              SeedIO sd;
+              sd.best = best;
+              E3_MAKE_CTX(ex);
+              seed_piece<DT, SAMPLER>(sd, ex, lane_data, e_lane, lim, sm);
+              best = sd.best;
+              R0 = sd.R0;
+            } else {
+              R0 = seed_reference<DT>(lane_data, e_lane, lim);
+            }
+            if (R0 > -CUDART_INF_F) {
+              const float nRc = -R0 * ri.c;
+              if (fabsf(nRc) < CUDART_INF_F) { acc.R = R0; acc.nRc = nRc; }
             }
             if (SAMPLER == 0) ethr = gate_threshold(best.enc, acc.nRc);
           } else if (SAMPLER == 0 && (c & 3) == 0) {
