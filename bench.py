@@ -47,7 +47,7 @@ METRIC = "logit rows/s, fused sample+entropy, V=151,936"
 UNIT = "rows/s"
 # dram__bytes_read.sum + dram__bytes_write.sum of one e3_sample launch of this workload (ncu capture summarised in
 # profiles/rows_kernel_c2_ncu_full.txt); only for the kernel variant that was captured.
-NCU_TRAFFIC_BYTES = {1: 161.5e6}
+NCU_TRAFFIC_BYTES = {1: 160.3e6}
 WORKLOAD = "rollout decode step: 512 rows (64 prompts x 8 rollouts) x V=151,936 bf16, 256 decode steps"
 
 
