@@ -43,6 +43,9 @@ __global__ void __launch_bounds__(kThreads) grpo_seq_kernel(const float *__restr
                                                             float *__restrict__ g_out, SeqPartial *__restrict__ part) {
   __shared__ double sh[kThreads / 32];
   __shared__ double s_gq;
+  // programmatic dependent launch: the final kernel may be set up while this one runs
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const int64_t i = blockIdx.x;
   const int64_t base = i * seq_len;
   if (threadIdx.x == 0) {
@@ -92,6 +95,7 @@ __global__ void __launch_bounds__(kThreads) grpo_final_kernel(const SeqPartial *
                                                               int64_t n_groups, double *__restrict__ out_J,
                                                               double *__restrict__ out_clip_frac) {
   __shared__ double sh[kThreads / 32];
+  asm volatile("griddepcontrol.wait;" ::: "memory");  // the per-response partials are complete and visible
   double J = 0.0, tok = 0.0, cl = 0.0;
   for (int64_t i = threadIdx.x; i < n_seq; i += kThreads) { J += part[i].J; tok += part[i].tokens; cl += part[i].clipped; }
   J = block_sum(J, sh);
@@ -125,10 +129,23 @@ extern "C" e3_status e3_grpo_objective(const float *logp, const float *logp_old,
   if (!workspace || workspace_bytes < e3::grpo_workspace_bytes(n_seq)) return E3_ERR_WORKSPACE;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   SeqPartial *part = static_cast<SeqPartial *>(workspace);
-  if (n_seq > 0)
-    grpo_seq_kernel<<<(unsigned)n_seq, kThreads, 0, s>>>(logp, logp_old, mask, seq_len, adv, group_offsets, n_groups,
-                                                         1.0 - (double)clip_eps, 1.0 + (double)clip_eps, out_g_logp,
-                                                         part);
-  grpo_final_kernel<<<1, kThreads, 0, s>>>(part, n_seq, n_groups, out_objective, out_clip_frac);
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t cfg = {};
+  cfg.blockDim = dim3(kThreads);
+  cfg.stream = s;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  if (n_seq > 0) {
+    cfg.gridDim = dim3((unsigned)n_seq);
+    if (cudaLaunchKernelEx(&cfg, grpo_seq_kernel, logp, logp_old, mask, seq_len, adv, group_offsets, n_groups,
+                           1.0 - (double)clip_eps, 1.0 + (double)clip_eps, out_g_logp, part) != cudaSuccess)
+      return E3_ERR_CUDA;
+  }
+  cfg.gridDim = dim3(1);
+  if (cudaLaunchKernelEx(&cfg, grpo_final_kernel, (const SeqPartial *)part, n_seq, n_groups, out_objective,
+                         out_clip_frac) != cudaSuccess)
+    return E3_ERR_CUDA;
   return cudaGetLastError() == cudaSuccess ? E3_OK : E3_ERR_CUDA;
 }
