@@ -360,3 +360,29 @@ def test_group_advantage_ragged(e3):
     adv, _ = e3.e3_group_advantage(r, off)
     radv, _ = oracle.group_advantage(r.cpu().numpy(), off.cpu().numpy())
     assert_close("adv.real", adv.cpu().numpy(), radv, 1e-5)
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_first_pieces_masked_or_invalid(e3, dtype):
+    """Every CTA's first row piece is masked out or has an unusable temperature (the finishing warp's dry run
+    then has nothing to walk through), in the split that cuts rows and in the one that hands out whole rows."""
+    V = 151936
+    for rows in (40, 1300):
+        logits = inputs.zipf_gaussian_logits(rows, V, seed=70 + rows, dtype=dtype, device=DEV)
+        targets = inputs.uniform_targets(rows, V, seed=71, device=DEV)
+        mask = torch.ones(rows, dtype=torch.uint8, device=DEV)
+        mask[::2] = 0
+        mask[: rows // 3] = 0
+        temps = inputs.uniform_temps(rows, seed=72, device=DEV)
+        temps[1::4] = float("nan")
+        lp, en = e3.e3_token_logp_entropy(logits, targets, mask=mask, temps=temps)
+        torch.cuda.synchronize()
+        rlp, ren, _ = oracle.token_logp_entropy(inputs.to_oracle_array(logits), targets.cpu().numpy(),
+                                                mask=mask.cpu().numpy(), temps=temps.cpu().numpy())
+        assert_close("logp", lp.cpu().numpy(), rlp, ATOL[dtype])
+        assert_close("ent", en.cpu().numpy(), ren, ATOL[dtype])
+        if rows == 40:
+            t2 = temps.clone()
+            t2[: rows // 2] = -1.0
+            for sampler in (0, 1):
+                _check_sample(e3, logits, t2, seed=5, counter=rows, sampler=sampler, name=f"s{sampler}")
