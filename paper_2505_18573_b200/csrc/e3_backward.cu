@@ -83,6 +83,10 @@ __global__ void __launch_bounds__(kThreads) backward_kernel(const BwdParams p) {
   constexpr int kVecE = DT == 0 ? 4 : 8;            // entries per 16-byte vector
   constexpr int kVecPerSeg = kSegE / kVecE;
   constexpr int kPerThread = kVecPerSeg / kThreads;  // 8 fp32 / 4 bf16 vectors per thread and item
+  // programmatic dependent launch: nothing in global memory is touched before the wait, which returns once
+  // the kernel before this one in the stream has completed
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   for (int64_t item = blockIdx.x; item < p.items; item += gridDim.x) {
     const int64_t row = item / p.segs_per_row;
     const int e0 = (int)((item - row * p.segs_per_row) * kSegE);
@@ -205,13 +209,17 @@ extern "C" e3_status e3_token_logp_entropy_backward(const void *logits, e3_dtype
   const unsigned grid = (unsigned)(p.items < cap ? p.items : cap);
   const bool aligned = !misaligned(logits, 16) && !misaligned(dlogits, 16) && (row_stride * esize) % 16 == 0 &&
                        (dlogits_stride * esize) % 16 == 0;
-  cudaStream_t s = static_cast<cudaStream_t>(stream);
-  if (dt == E3_F32) {
-    if (aligned) backward_kernel<0, true><<<grid, kThreads, 0, s>>>(p);
-    else backward_kernel<0, false><<<grid, kThreads, 0, s>>>(p);
-  } else {
-    if (aligned) backward_kernel<1, true><<<grid, kThreads, 0, s>>>(p);
-    else backward_kernel<1, false><<<grid, kThreads, 0, s>>>(p);
-  }
-  return cudaGetLastError() == cudaSuccess ? E3_OK : E3_ERR_CUDA;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(kThreads);
+  cfg.stream = static_cast<cudaStream_t>(stream);
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  cudaError_t e;
+  if (dt == E3_F32) e = aligned ? cudaLaunchKernelEx(&cfg, backward_kernel<0, true>, p) : cudaLaunchKernelEx(&cfg, backward_kernel<0, false>, p);
+  else e = aligned ? cudaLaunchKernelEx(&cfg, backward_kernel<1, true>, p) : cudaLaunchKernelEx(&cfg, backward_kernel<1, false>, p);
+  return e == cudaSuccess ? E3_OK : E3_ERR_CUDA;
 }
