@@ -21,14 +21,19 @@
 // wait runs out the CTA stops waiting altogether, finishes its fixed sequence of steps on whatever
 // data it has and marks its rows invalid.  The kernel is launched with programmatic stream
 // serialization: its set-up overlaps the tail of the kernel before it in the stream, and it touches
-// global memory only after griddepcontrol.wait.
+// global memory only after griddepcontrol.wait.  The finishing warp walks through its own code once
+// while the first piece streams (a dry run without side effects), because that code runs last in the
+// CTA's life and a first run through cold instructions took several times as long as a warm one.
 //
 // Numerics.  All lanes of a warp share a reference logit R; each thread keeps the sums Z = sum 2^t,
 // W = sum 2^t * t with t = z*c - R*c and c = log2(e)/tau, two entries per instruction (packed fp32).
 // The streaming loop never looks for the maximum: R is taken from the first entries of the row piece;
-// when the sum of a group of 16 leaves the safe range (some t above 1..5) the warp moves R up to the
-// largest logit of the current turn, rescales its sums and repeats the group.  R therefore stays
-// close to the largest logit seen, which keeps W/Z small and the entropy free of cancellation.
+// the sums of a turn stay local until the warp has checked them, and when one leaves the safe range
+// (some t above 1..5) the warp moves R up to the largest logit of the current turn, rescales its state
+// and repeats the turn.  R therefore stays close to the largest logit seen, which keeps W/Z small and
+// the entropy free of cancellation.  A turn is the thread's 64 bytes of a stage in straight-line code
+// when the stage lies wholly inside the row and sampler 0's per-group work is not needed, otherwise
+// a group of 16 entries.
 // -inf logits are clamped to a huge negative finite value on the way in, which gives them weight 0
 // without special cases; NaN and +inf end up in a careful out-of-line form that flags the row.
 // States merge associatively; the per-row result is formed in fp64:
@@ -45,8 +50,10 @@
 // whole row again when there are three or more).  The token never depends on the gating or on fp32.
 //
 // Sampler 1 (one Gumbel per block of 256 entries).  8 (bf16) or 16 (fp32) neighbouring lanes hold
-// one block per step; their sums are added with shuffles, each lane parks one block and all lanes
-// score their parked blocks together.
+// one block per step; every lane writes its sum to a per-warp scratch in shared memory, and every
+// 8 / 16 steps lane j of each group adds up the block of step j and all lanes score their blocks
+// together (fp32, three leaders per thread).  The finishing warp settles near-ties of block scores in
+// fp64 and draws inside the winning block by inverse CDF (fp32, fp64 near a prefix boundary).
 #include "e3_rows.cuh"
 
 #include <limits.h>
