@@ -13,14 +13,29 @@
  *
  * Conventions for every device call
  *   - "device" pointers are CUDA device pointers owned by the caller; the
- *     library allocates and frees nothing and keeps no state between calls.
+ *     library allocates and frees no device memory.  What it keeps between calls, per process:
+ *     a counter that gives every row call its own id (the tag of the partial row states in the
+ *     workspace), a per-device record of each kernel's launch set-up (filled on first use), and
+ *     for e3_masked_mean_entropy_static the address of its built-in scratch.  No result depends on them.
+ *   - Pointers: every pointer must be aligned to its element type (else E3_ERR_ALIGNMENT);
+ *     workspaces to 16 bytes.  Optional outputs are NULL when not wanted.
  *   - Work is enqueued on `stream` (a cudaStream_t passed as void*; NULL = the
- *     legacy default stream).  Calls never synchronise, print or abort.
+ *     legacy default stream).  Calls never synchronise, print or abort.  The kernels are launched with
+ *     programmatic stream serialization: their set-up may overlap the tail of the work before them in
+ *     the stream; they touch memory only after that work has completed.
  *   - The return value reports what the host can see (bad sizes, NULL
  *     pointers, launch failure).  Problems only the device can see (NaN or
  *     +inf logit, a row of -inf only, tau < 0 or not finite) mark that row:
- *     token -1, log-prob and entropy NaN.  Other rows are unaffected.
+ *     token -1, log-prob, entropy and gap NaN.  Other rows are unaffected.
+ *   - Every wait inside a kernel is bounded (two seconds).  If one ever runs out, the thread block
+ *     concerned gives up: its unfinished rows read token -1 / NaN and bit E3_STATUS_TIMEOUT is OR-ed
+ *     into the caller's status word (`out_status`, optional, never cleared by the library).  The host
+ *     sees it after synchronising; e3_status has E3_ERR_TIMEOUT for callers that want to pass it on.
+ *     After a timeout, clear a workspace (cudaMemsetAsync) before a captured graph that uses it is
+ *     replayed.
  *   - Results are bit-reproducible for identical arguments.
+ *   - Stream capture: every call may be captured into a CUDA graph and replayed (the row calls wipe
+ *     their partial row states when a row is finished, so a replay never meets an old one).
  *   - rows == 0 / n == 0 / n_groups == 0 are valid no-ops.
  */
 #ifndef E3_H_
@@ -47,8 +62,12 @@ typedef enum {
   E3_ERR_WORKSPACE = 4,   /* workspace missing or smaller than e3_workspace_bytes() says */
   E3_ERR_INFEASIBLE = 5,  /* Algorithm 1: needs G_min <= G <= G_max */
   E3_ERR_CUDA = 6,        /* a CUDA runtime call failed (no device, launch error) */
-  E3_ERR_TIMEOUT = 7      /* reserved: a bounded device-side wait ran out */
+  E3_ERR_TIMEOUT = 7      /* a bounded device-side wait ran out: never returned by a call (calls do not
+                             synchronise); the code for a caller that found E3_STATUS_TIMEOUT in its status word */
 } e3_status;
+
+/* Bits of the device status word (`out_status` of the row calls). */
+#define E3_STATUS_TIMEOUT 1
 
 typedef enum { E3_F32 = 0, E3_BF16 = 1 } e3_dtype;
 
@@ -77,7 +96,9 @@ E3_API const char *e3_status_string(e3_status s);
 
 /* Bytes of device scratch a call uses for the given problem size.  For
  * E3_CALL_MASKED_MEAN_ENTROPY `rows` is the number of tokens n, for E3_CALL_GRPO_OBJECTIVE the number of
- * responses n_seq; V, dt are ignored for both.
+ * responses n_seq; V, dt are ignored for both.  E3_CALL_SAMPLE: 256 KiB for the partial states of cut rows plus,
+ * for E3_SAMPLER_BLOCK, the per-lane sums the second kernel reads (about 1/32 of the bytes of the logits);
+ * E3_CALL_TOKEN_LOGP_ENTROPY: 256 KiB plus the partial sums of the fused mean entropy.
  * Scratch contents on entry never matter.  A workspace must not be shared by calls that can run
  * at the same time (different streams without ordering).  It must be 16-byte aligned. */
 E3_API size_t e3_workspace_bytes(e3_call which, int64_t rows, int64_t V, e3_dtype dt);
@@ -103,16 +124,24 @@ E3_API size_t e3_workspace_bytes(e3_call which, int64_t rows, int64_t V, e3_dtyp
  *               ties go to the lower index.
  *               Sampler 1: u_b = (x_b + 1/2) 2^-32, x_b word (b mod 4) of call b/4 of stream 2, for block b;
  *               the in-block draw uses word 0 of call 0 of stream 3.
+ *               row_base >= 0 and row_base + rows <= 2^32 (the row number is one 32-bit counter word), else
+ *               E3_ERR_INVALID_ARG.
  *   out_tok     device int32 [rows], required.   out_logp, out_ent: device float [rows], each may be NULL.
+ *   out_gap     device float [rows] or NULL: the mean logit gap of App. A in units of tau,
+ *               beta sum_i p_i Delta_i with Delta_i = z_max - z_i (so that H = ln sum_i exp(-beta Delta_i) + gap);
+ *               0 for greedy rows.  Asking for it selects a kernel variant that also tracks z_max.
+ *   out_status  device int32 or NULL: status word, see the conventions above.
  *   workspace   device scratch of e3_workspace_bytes(E3_CALL_SAMPLE, ...) bytes.  It holds the partial states
  *               of rows that are split between thread blocks so that every block streams the same number
- *               of bytes.  NULL (or too small) is accepted: rows are then never split, which costs
- *               throughput when there are fewer than a few thousand rows.
+ *               of bytes, and what the two kernels of E3_SAMPLER_BLOCK hand to each other.  For the other
+ *               samplers NULL (or fewer than 256 KiB) is accepted: rows are then never split, which costs
+ *               throughput when there are fewer than a few thousand rows.  E3_SAMPLER_BLOCK needs the full
+ *               size (E3_ERR_WORKSPACE).
  * -inf logits are allowed (probability 0, never drawn).
  */
 E3_API e3_status e3_sample(const void *logits, e3_dtype dt, int64_t rows, int64_t V, int64_t row_stride,
                     const float *temps, uint64_t seed, uint64_t counter, int64_t row_base, e3_sampler sampler,
-                    int32_t *out_tok, float *out_logp, float *out_ent,
+                    int32_t *out_tok, float *out_logp, float *out_ent, float *out_gap, int32_t *out_status,
                     void *workspace, size_t workspace_bytes, void *stream);
 
 /*
@@ -124,13 +153,22 @@ E3_API e3_status e3_sample(const void *logits, e3_dtype dt, int64_t rows, int64_
  * logits are not read.  A target outside [0, V) gives out_logp = NaN (entropy still valid).
  *
  *   targets     device int32 [rows];  mask: device uint8 [rows] or NULL (= all ones)
- *   out_logp, out_ent   device float [rows], each may be NULL
+ *   out_logp, out_ent, out_gap   device float [rows], each may be NULL (out_gap as in e3_sample; 0 on masked rows)
+ *   out_ent_sum, out_count   both NULL, or both device double scalars: the batch entropy of the scheduler
+ *               (Sec. 4.2) from the same call: out_ent_sum = sum_r mask[r] out_ent[r] accumulated in fp64 in
+ *               the fixed order of e3_masked_mean_entropy, out_count = sum_r mask[r]; out_ent_sum / out_count
+ *               equals that call's mean bit for bit.  Needs out_ent and the workspace
+ *               (E3_ERR_INVALID_ARG / E3_ERR_WORKSPACE).  The reduction runs as two small kernels behind
+ *               the row kernel, chained by programmatic dependent launch.
+ *   workspace   e3_workspace_bytes(E3_CALL_TOKEN_LOGP_ENTROPY, rows, V, dt) bytes; NULL or fewer than
+ *               256 KiB is accepted when the fused mean is not asked for (rows are then never split).
  * Other arguments as in e3_sample.
  */
 E3_API e3_status e3_token_logp_entropy(const void *logits, e3_dtype dt, int64_t rows, int64_t V, int64_t row_stride,
                                 const int32_t *targets, const uint8_t *mask,
                                 const float *temps, float temp_scalar,
-                                float *out_logp, float *out_ent,
+                                float *out_logp, float *out_ent, float *out_gap,
+                                double *out_ent_sum, double *out_count, int32_t *out_status,
                                 void *workspace, size_t workspace_bytes, void *stream);
 
 /*
@@ -204,8 +242,8 @@ E3_API e3_status e3_masked_mean_entropy_static(const float *ent, const uint8_t *
  * [group_offsets[g], group_offsets[g+1]):  A_i = (r_i - mean) / (std + eps).
  * Groups may have any size (the rollout budget of Algorithm 1 makes them ragged).
  * std is the sample standard deviation (divide by n-1) when unbiased != 0, else the population one.
- * eps > 0 makes a group with identical rewards give exactly 0, as Sec. 4.2 assumes.
- * A group of one gives 0; an empty group writes nothing.
+ * A group with identical rewards gives exactly 0, as Sec. 4.2 assumes (also with eps == 0, where the
+ * quotient would be 0/0).  eps must be >= 0 and finite.  A group of one gives 0; an empty group writes nothing.
  *
  *   rewards        device float [group_offsets[n_groups]]
  *   group_offsets  device int64 [n_groups + 1], non-decreasing, [0] == 0
@@ -321,6 +359,15 @@ E3_API e3_status e3_update_temperature_gap(e3_sched *s, double H_t, double *tau_
 
 /* Target entropy the scheduler holds at step s->t (H_init before annealing starts). */
 E3_API double e3_anneal_target(const e3_sched *s);
+
+/*
+ * Test hook, not for production use.  The next row call of this process (e3_sample or
+ * e3_token_logp_entropy) leaves the 4 KiB tile number `tile` of its logits (row * ceil(V * esize / 4096)
+ * + tile within the row) uncopied, and its waits give up after wait_ns nanoseconds instead of two seconds.
+ * The consumer of that tile then runs into the bounded wait: the call returns as usual, the rows of the
+ * thread block concerned read token -1 / NaN, and E3_STATUS_TIMEOUT appears in the status word.  One shot.
+ */
+E3_API void e3_test_arm_stall(int64_t tile, uint64_t wait_ns);
 
 #ifdef __cplusplus
 }

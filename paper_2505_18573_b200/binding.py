@@ -16,6 +16,8 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "libe3.so")
 
 E3_OK = 0
+E3_ERR_INVALID_ARG, E3_ERR_DTYPE, E3_ERR_ALIGNMENT, E3_ERR_WORKSPACE, E3_ERR_INFEASIBLE, E3_ERR_CUDA, E3_ERR_TIMEOUT = 1, 2, 3, 4, 5, 6, 7
+E3_STATUS_TIMEOUT = 1
 E3_F32, E3_BF16 = 0, 1
 E3_SAMPLER_TOKEN, E3_SAMPLER_BLOCK, E3_SAMPLER_TOKEN_AUDIT = 0, 1, 2
 E3_CALL_SAMPLE, E3_CALL_TOKEN_LOGP_ENTROPY, E3_CALL_MASKED_MEAN_ENTROPY, E3_CALL_GRPO_OBJECTIVE = 0, 1, 2, 3
@@ -24,7 +26,8 @@ E3_SAMPLE_BLOCK = 256
 EXPORTS = ("e3_status_string", "e3_workspace_bytes", "e3_sample", "e3_token_logp_entropy",
            "e3_token_logp_entropy_backward", "e3_grpo_objective",
            "e3_masked_mean_entropy", "e3_masked_mean_entropy_static", "e3_group_advantage", "e3_allocate_budget", "e3_update_temperature",
-           "e3_anneal_target", "e3_entropy_gap", "e3_update_temperature_gap", "e3_difficulty_accumulate", "e3_difficulty_rank", "e3_budget_curriculum")
+           "e3_anneal_target", "e3_entropy_gap", "e3_update_temperature_gap", "e3_difficulty_accumulate", "e3_difficulty_rank", "e3_budget_curriculum",
+           "e3_test_arm_stall")
 
 
 class E3Error(RuntimeError):
@@ -57,11 +60,11 @@ def lib() -> C.CDLL:
         L.e3_sample.restype = C.c_int
         L.e3_sample.argtypes = [C.c_void_p, C.c_int, C.c_int64, C.c_int64, C.c_int64, C.c_void_p, C.c_uint64,
                                 C.c_uint64, C.c_int64, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
-                                C.c_size_t, C.c_void_p]
+                                C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
         L.e3_token_logp_entropy.restype = C.c_int
         L.e3_token_logp_entropy.argtypes = [C.c_void_p, C.c_int, C.c_int64, C.c_int64, C.c_int64, C.c_void_p,
                                             C.c_void_p, C.c_void_p, C.c_float, C.c_void_p, C.c_void_p, C.c_void_p,
-                                            C.c_size_t, C.c_void_p]
+                                            C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
         L.e3_token_logp_entropy_backward.restype = C.c_int
         L.e3_token_logp_entropy_backward.argtypes = [C.c_void_p, C.c_int, C.c_int64, C.c_int64, C.c_int64, C.c_void_p,
                                                      C.c_void_p, C.c_void_p, C.c_float, C.c_void_p, C.c_void_p,
@@ -97,6 +100,8 @@ def lib() -> C.CDLL:
                                            C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
         L.e3_anneal_target.restype = C.c_double
         L.e3_anneal_target.argtypes = [C.POINTER(e3_sched)]
+        L.e3_test_arm_stall.restype = None
+        L.e3_test_arm_stall.argtypes = [C.c_int64, C.c_uint64]
         _lib = L
     return _lib
 
@@ -161,10 +166,18 @@ def _row_workspace(device, stream_handle: int, which: int, rows: int, V: int, dt
     return ws
 
 
+def _status_word(status):
+    if status is not None and (not status.is_cuda or status.dtype != torch.int32 or status.numel() < 1):
+        raise ValueError("status must be an int32 CUDA tensor")
+    return status
+
+
 def e3_sample(logits, temps, seed: int, counter: int, row_base: int = 0, sampler: int = E3_SAMPLER_TOKEN,
               out_tok=None, out_logp=None, out_ent=None, want_logp: bool = True, want_ent: bool = True,
-              workspace=None, stream=None):
-    """Rollout step: returns (tok int32, logp float32 | None, ent float32 | None), each [rows]."""
+              out_gap=None, want_gap: bool = False, status=None, workspace=None, stream=None):
+    """Rollout step: returns (tok int32, logp float32 | None, ent float32 | None), each [rows]; with
+    ``want_gap`` or ``out_gap`` a fourth element, the mean logit gap float32 [rows].  ``status``: optional
+    int32 CUDA tensor, the device status word (E3_STATUS_TIMEOUT is OR-ed in, never cleared)."""
     dt, rows, V, stride = _logits_desc(logits)
     _dev(temps, "temps")
     if temps.dtype != torch.float32 or temps.numel() != rows or not temps.is_contiguous():
@@ -176,19 +189,27 @@ def e3_sample(logits, temps, seed: int, counter: int, row_base: int = 0, sampler
         out_logp = torch.empty(rows, dtype=torch.float32, device=dev)
     if out_ent is None and want_ent:
         out_ent = torch.empty(rows, dtype=torch.float32, device=dev)
+    if out_gap is None and want_gap:
+        out_gap = torch.empty(rows, dtype=torch.float32, device=dev)
     sh = _stream(stream)
     if workspace is None:
         workspace = _row_workspace(dev, sh, E3_CALL_SAMPLE, rows, V, dt)
     st = lib().e3_sample(_ptr(logits), dt, rows, V, stride, _ptr(temps), seed, counter, row_base, sampler,
-                         _ptr(out_tok), _ptr(out_logp), _ptr(out_ent), _ptr(workspace),
-                         workspace.numel() * workspace.element_size(), sh)
+                         _ptr(out_tok), _ptr(out_logp), _ptr(out_ent), _ptr(out_gap), _ptr(_status_word(status)),
+                         _ptr(workspace), workspace.numel() * workspace.element_size(), sh)
     _check("e3_sample", st)
+    if out_gap is not None:
+        return out_tok, out_logp, out_ent, out_gap
     return out_tok, out_logp, out_ent
 
 
 def e3_token_logp_entropy(logits, targets, mask=None, temps=None, temp_scalar: float = 1.0, out_logp=None,
-                          out_ent=None, workspace=None, stream=None):
-    """Training-side pass: returns (logp float32, ent float32), each [rows]; masked rows give 0."""
+                          out_ent=None, out_gap=None, want_gap: bool = False, out_sum=None, status=None,
+                          workspace=None, stream=None):
+    """Training-side pass: returns (logp float32, ent float32), each [rows]; masked rows give 0.  With
+    ``want_gap`` or ``out_gap`` a third element, the mean logit gap float32 [rows].  ``out_sum``: optional
+    float64 CUDA tensor [2] that receives (sum of entropies over unmasked rows, their number), the fused
+    batch entropy.  ``status``: optional int32 CUDA tensor, the device status word."""
     dt, rows, V, stride = _logits_desc(logits)
     _dev(targets, "targets"); _dev(mask, "mask"); _dev(temps, "temps")
     if targets.dtype != torch.int32 or targets.numel() != rows:
@@ -202,13 +223,22 @@ def e3_token_logp_entropy(logits, targets, mask=None, temps=None, temp_scalar: f
         out_logp = torch.empty(rows, dtype=torch.float32, device=dev)
     if out_ent is None:
         out_ent = torch.empty(rows, dtype=torch.float32, device=dev)
+    if out_gap is None and want_gap:
+        out_gap = torch.empty(rows, dtype=torch.float32, device=dev)
+    if out_sum is not None and (not out_sum.is_cuda or out_sum.dtype != torch.float64 or out_sum.numel() != 2
+                                or not out_sum.is_contiguous()):
+        raise ValueError("out_sum must be a contiguous float64 CUDA tensor with two entries")
     sh = _stream(stream)
     if workspace is None:
         workspace = _row_workspace(dev, sh, E3_CALL_TOKEN_LOGP_ENTROPY, rows, V, dt)
+    sum_ptr = None if out_sum is None else out_sum.data_ptr()
     st = lib().e3_token_logp_entropy(_ptr(logits), dt, rows, V, stride, _ptr(targets), _ptr(mask), _ptr(temps),
-                                     float(temp_scalar), _ptr(out_logp), _ptr(out_ent), _ptr(workspace),
-                                     workspace.numel() * workspace.element_size(), sh)
+                                     float(temp_scalar), _ptr(out_logp), _ptr(out_ent), _ptr(out_gap), sum_ptr,
+                                     None if sum_ptr is None else sum_ptr + 8, _ptr(_status_word(status)),
+                                     _ptr(workspace), workspace.numel() * workspace.element_size(), sh)
     _check("e3_token_logp_entropy", st)
+    if out_gap is not None:
+        return out_logp, out_ent, out_gap
     return out_logp, out_ent
 
 
@@ -395,3 +425,8 @@ def e3_budget_curriculum(G: int, step: int, G_min_limit: int, G_max_limit: int, 
     _check("e3_budget_curriculum", st)
     return lo.value, hi.value
 
+
+
+def e3_test_arm_stall(tile: int, wait_ns: int) -> None:
+    """Test hook: the next row call leaves one 4 KiB tile uncopied and bounds its waits by ``wait_ns``."""
+    lib().e3_test_arm_stall(int(tile), int(wait_ns))

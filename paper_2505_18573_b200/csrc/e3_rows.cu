@@ -1,59 +1,70 @@
-// Row-streaming kernel: one pass over the logits of a row gives the softmax statistics
+// Row-streaming kernels: one pass over the logits of a row gives the softmax statistics
 // (App. A: Z(beta), Eq. "entropy" in its shifted form H = ln Z + beta sum p_i Delta_i), the
 // log-probability of one token and, for rollouts, a Gumbel-max sample.
 //
-// Work split.  The [rows, V] matrix is cut into tiles of 512 entries and every CTA of a
-// persistent grid (two per SM) takes an equal, contiguous run of tiles, so all CTAs stream the
-// same number of bytes whatever the number of rows.  A run covers the tail of one row, some
-// whole rows and the head of another.  Whole rows are finished by the CTA itself.  For a row
-// that is cut, every CTA holding a piece stores its partial state in the caller's workspace (64-bit
-// words tagged with a per-call id), issues a sequentially consistent fence and then looks for the
-// row's other pieces: the CTA whose fence comes last finds them all, merges them and writes the
-// outputs.  Nobody waits for anybody.  (With a response mask, and when no workspace is given, CTAs
-// take whole rows round-robin instead.)
+// Work split.  A row is cut into tiles of 4 KiB of logits and every CTA of a persistent grid (two per
+// SM) takes an equal, contiguous run of tiles, so all CTAs stream the same number of bytes whatever
+// the number of rows.  A run covers the tail of one row, some whole rows and the head of another; a
+// CTA works on its two cut pieces first and on its whole rows last, so that what is left to do at
+// the end of its life is the cheap finish of a row it holds alone.  For a row that is cut, a CTA first
+// looks (while its consumers are still streaming, and again when they are done) whether the row's other
+// pieces are in the caller's workspace already; if so it is the last to arrive and finishes the row
+// without publishing anything.  Otherwise it stores its partial state (64-bit words tagged with a
+// per-call id), issues a sequentially consistent fence and looks once more: of all CTAs that hold a
+// piece, the one whose fence comes last finds them all.  Whoever finishes a row merges the pieces in
+// piece order, writes the outputs and wipes the tags of the pieces it used, so that a replay of the
+// same launch (a captured graph) never meets a piece of an earlier run.  Nobody waits for anybody.
+// (With a response mask over many rows, and when no workspace is given, CTAs take whole rows
+// round-robin instead.)
 //
-// Inside a CTA: one thread issues bulk asynchronous copies (cp.async.bulk, no multicast) of 16 KiB
-// into a 4-stage shared-memory ring guarded by mbarriers; eight warps consume the ring, each
-// thread 64 contiguous bytes per stage (read in a swizzled vector order that is free of bank
-// conflicts); one warp finishes rows (merges the eight warp states, fp64 epilogue, piece protocol)
-// so that the consumers never stall on it.  Consumers and the finishing warp look one row ahead for
-// the temperature; the copy-issuing thread never needs it.  Every mbarrier wait is bounded: when a
-// wait runs out the CTA stops waiting altogether, finishes its fixed sequence of steps on whatever
-// data it has and marks its rows invalid.  The kernel is launched with programmatic stream
-// serialization: its set-up overlaps the tail of the kernel before it in the stream, and it touches
-// global memory only after griddepcontrol.wait.  The finishing warp walks through its own code once
-// while the first piece streams (a dry run without side effects), because that code runs last in the
-// CTA's life and a first run through cold instructions took several times as long as a warm one.
+// Inside a CTA.  Each of the eight consumer warps owns a ring of three 4 KiB slots.  One warp feeds
+// the rings, lane w feeding consumer warp w: per slot one bulk asynchronous copy (cp.async.bulk with a
+// plain, CTA-local shared-memory destination, completion counted in bytes on the slot's mbarrier), a
+// 4-byte asynchronous copy of the row's temperature that completes on the same barrier, and a small
+// record that says what the slot holds (row, first entry, number of entries, first/last slice of a row
+// piece).  The consumers keep no position of their own: every slot describes itself.  Consumer warp w
+// takes tiles w, w + 8, ... of a piece.  A consumer thread takes 128 contiguous bytes of a slot, read as
+// 16-byte vectors in the order i xor (lane mod 8), which keeps the eight lanes of a quarter warp on
+// distinct banks.  One more warp finishes rows (merges the eight warp states, fp64 epilogue, piece
+// protocol, sampler 0's settling of near-ties) so that the consumers never stall on it.
+// Every wait is bounded in time: when one runs out the CTA stops waiting altogether, marks the rows it
+// has not finished as invalid (token -1, NaN), sets the timeout bit of the caller's status word, sees
+// its copies in flight land (bounded again) and returns.  The kernels are launched with programmatic
+// stream serialization: their set-up overlaps the tail of the kernel before them in the stream, and
+// they touch global memory only after griddepcontrol.wait.
 //
 // Numerics.  All lanes of a warp share a reference logit R; each thread keeps the sums Z = sum 2^t,
 // W = sum 2^t * t with t = z*c - R*c and c = log2(e)/tau, two entries per instruction (packed fp32).
-// The streaming loop never looks for the maximum: R is taken from the first entries of the row piece;
-// the sums of a turn stay local until the warp has checked them, and when one leaves the safe range
-// (some t above 1..5) the warp moves R up to the largest logit of the current turn, rescales its state
-// and repeats the turn.  R therefore stays close to the largest logit seen, which keeps W/Z small and
-// the entropy free of cancellation.  A turn is the thread's 64 bytes of a stage in straight-line code
-// when the stage lies wholly inside the row and sampler 0's per-group work is not needed, otherwise
-// a group of 16 entries.
-// -inf logits are clamped to a huge negative finite value on the way in, which gives them weight 0
-// without special cases; NaN and +inf end up in a careful out-of-line form that flags the row.
-// States merge associatively; the per-row result is formed in fp64:
-// H = ln Z - ln2 * W / Z,  ln p_tok = (z_tok*c - M) ln2 - ln Z.
+// The streaming loop never looks for the maximum: the sums of a turn (the thread's 128 bytes of a
+// slot) stay local until the warp has checked them with one vote, and when one leaves the safe range
+// (some t above 7, a NaN, an infinity) nothing has been added yet and the turn is taken again by the
+// careful form, which moves R up to the largest logit of the slot, rescales the state, skips -inf
+// entries and flags NaN and +inf.  R therefore stays close to the largest logit seen, which keeps W/Z
+// small and the entropy free of cancellation.  States merge associatively; the per-row result is
+// formed in fp64:  H = ln Z - ln2 * W / Z,  ln p_tok = (z_tok*c - M) ln2 - ln Z, and, where the caller
+// asks for it, the mean logit gap beta sum p_i Delta_i = (z_max*c - M - W/Z) ln2 of App. A (this variant
+// of the kernel also tracks the largest logit, half an instruction per entry more).
 //
 // Sampler 0 (one Gumbel per vocabulary entry).  u_i has 8 coarse + 32 fine bits.  An entry can
 // only win if its coarse byte is 255 (g_i >= 5.5432) or if z_i/tau exceeds the best score so
-// far minus 5.5432; the second condition is tested on the group sum of 2^t, which bounds every
-// term from above.  Groups that pass are copied (coarse bytes and logits) into a per-warp queue
-// in shared memory with ballot-compacted positions; when 32 are waiting the warp scores them, one
+// far minus 5.5432; the second condition is tested on the sum of 2^t over the entry's group of 16,
+// which bounds every term from above.  Groups that pass are copied into a per-warp queue in shared
+// memory with ballot-compacted positions; when enough are waiting the warp scores them, one group
 // per lane, in fp32 with a proven error bound, and every thread keeps its three leaders.  The
 // finishing warp takes the fp32 leader when it is ahead by more than two error bounds; otherwise
 // it evaluates the contenders in fp64 with the expression order of the definition (or looks at the
 // whole row again when there are three or more).  The token never depends on the gating or on fp32.
 //
-// Sampler 1 (one Gumbel per block of 256 entries).  8 (bf16) or 16 (fp32) neighbouring lanes hold
-// one block per step; every lane writes its sum to a per-warp scratch in shared memory, and every
-// 8 / 16 steps lane j of each group adds up the block of step j and all lanes score their blocks
-// together (fp32, three leaders per thread).  The finishing warp settles near-ties of block scores in
-// fp64 and draws inside the winning block by inverse CDF (fp32, fp64 near a prefix boundary).
+// Sampler 1 (one Gumbel per block of 256 entries) is two kernels.  The consumers of the streaming kernel
+// do nothing for it but one shared-memory store per turn: every lane leaves its sum of 2^t over its 128
+// bytes (4 or 8 neighbouring lanes make up a block) and lane 0 the reference the sums refer to in a
+// 144-byte record next to the rings; the feeding lane ships the record to the caller's workspace with a
+// bulk asynchronous store when it sees the slot freed.  (A global store from a consumer costs the warp
+// microseconds while the copies keep the memory system busy, and so does every instruction-cache miss:
+// whatever the consumers execute besides their loop is dear.)  block_sample_kernel, launched behind the
+// streaming kernel, adds the lanes of every block, turns the sums into scores L_b + g_b (fp32, three
+// leaders per thread), settles near-ties of block scores in fp64 and draws inside the winning block by
+// inverse CDF (fp32, fp64 near a prefix boundary).  The workspace traffic is 1/28 of the logits.
 #include "e3_rows.cuh"
 
 #include <limits.h>
@@ -70,11 +81,7 @@ namespace {
 using u64 = unsigned long long;
 using f2 = float2;  // two fp32 values in a register pair
 
-constexpr int kQueueCap = 64;   // candidate groups a warp can hold
-constexpr int kDrainAt = 32;    // ... and the fill at which it evaluates them (one per lane)
-constexpr int kQueueHdrBytes = kQueueCap * 4;
 constexpr int kSlots = 4;  // hand-over slots between the consumer warps and the finishing warp
-constexpr uint32_t kSpinLimit = 1u << 23;  // polls before a wait gives up (seconds)
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2f = 0.6931471805599453f;
 constexpr double kLn2 = 0.6931471805599453094;
@@ -82,28 +89,40 @@ constexpr double kLn2 = 0.6931471805599453094;
 // with all 40 bits set the largest value is -ln(-ln(1 - 2^-41)) = 28.41903...  Both rounded up.
 constexpr float kGumbelCapCoarse = 5.5433f;
 constexpr float kGumbelCapAll = 28.4192f;
-// A group of 16 whose sum of 2^t is above this (or NaN) means that the warp's reference logit is stale:
-// the warp moves it up to the largest logit of the current turn and repeats the group.  Every entry that
-// is added therefore has t <= 5 while the reference is a logit the warp has really seen, so W/Z stays
-// small and the entropy ln Z - ln2 W/Z is free of cancellation at the 1e-5 level.
-constexpr float kGroupSumMax = 32.f;
-// Logits below this (also -inf) enter the streaming form as this value: weight 2^-huge = 0.
-constexpr uint32_t kFloorBf16x2 = 0xF180F180u;  // -2^100 twice
-constexpr float kFloorF32 = -1.2676506e30f;     // -2^100
+// A turn (up to 64 entries of one thread) whose sum of 2^t is above this (or NaN) means that the warp's
+// reference logit is stale: every entry that is added has t <= 7 while the reference is a logit the
+// warp has really seen, so W/Z stays small and the entropy ln Z - ln2 W/Z is free of cancellation at the
+// 1e-5 level.  (64 entries equal to the reference give 64: a flat row must pass.)
+constexpr float kTurnSumMax = 128.f;
+constexpr float kTurnWMax = 1e30f;  // |sum 2^t t| of a sound turn stays far below (a -inf logit makes it NaN)
+constexpr float kNoRef = 1e30f;     // nRc of a state without reference: the first turn overflows into the careful form
 
 enum : int { kErrValue = 1, kErrTimeout = 4 };
+enum : uint32_t { kFlagFirst = 1u, kFlagLast = 2u, kFlagEnd = 8u };
 
 template <int DT>
 struct Fmt {
   static constexpr int kEsize = DT == 0 ? 4 : 2;
-  static constexpr int kLaneE = kLaneBytes / kEsize;          // entries per thread and stage: 16 fp32 / 32 bf16
-  static constexpr int kG = kLaneE / kGroup;                  // groups per thread and stage: 1 / 2
-  static constexpr int kVG = 4 / kG;                          // 16-byte vectors per group: 4 / 2
-  static constexpr int kChunkE = kStageBytes / kEsize;        // entries per stage: 4,096 / 8,192
-  static constexpr int kEntryBytes = 16 + kGroup * kEsize;    // queue entry: coarse bytes + logits of one group
-  static constexpr int kQueueBytes = kQueueHdrBytes + kQueueCap * kEntryBytes;
-  static constexpr int kLB = 256 / kLaneE;                    // lanes that hold one block of sampler 1: 16 / 8
+  static constexpr int kLaneE = kLaneBytes / kEsize;  // entries per thread and stage: 32 fp32 / 64 bf16
+  static constexpr int kWarpE = 32 * kLaneE;          // entries per warp and stage = entries per tile: 1,024 / 2,048
+  static constexpr int kStageE = kStreamWarps * kWarpE;  // entries per stage: 8,192 / 16,384
+  static constexpr int kVG = kEsize;                  // 16-byte vectors per group of 16 entries: 4 / 2
+  static constexpr int kG = 8 / kVG;                  // groups per thread and stage: 2 / 4
+  static constexpr int kLB = 256 / kLaneE;            // lanes that hold one block of sampler 1: 8 / 4
+  static constexpr int kEntryBytes = kGroup * kEsize; // queue entry of sampler 0: the logits of one group
 };
+
+// Sampler 0 queues: a push never meets a queue holding kDrainAt or more groups and adds at most 32.
+constexpr int kDrainAt = 16;
+constexpr int kQueueCap = kDrainAt + 32;
+template <int DT>
+struct QueueBytes { static constexpr int value = kQueueCap * 4 + kQueueCap * Fmt<DT>::kEntryBytes; };
+// fp32 logits with sampler 0 need the larger queue entries: two ring stages there (the variant is bound
+// by the per-entry random numbers, not by the copies in flight)
+template <int DT, int SAMPLER>
+struct RingStages { static constexpr int value = (DT == 0 && SAMPLER == 0) ? 2 : kStages; };
+// Sampler 1: per consumer warp two records (144 bytes) per ring slot, used alternately, behind the rings.
+constexpr int kRecordBytesPerWarp = 2 * kStages * kRecordFloats * 4;
 
 // One partial row state.  In the workspace it is kPieceWords 64-bit words, each (tag << 32 | payload):
 // the tag depends on the call and on the word, so a reader knows word by word whether what it sees was
@@ -112,7 +131,7 @@ struct Piece {
   float M, Z, W;   // reference (log2 units), sum 2^t, sum 2^t t
   float zf;        // sampler 0: logit of entry tb[0]
   int err;
-  int pad;
+  float zmax;      // largest logit (only where the mean logit gap is asked for)
   float ty[3];     // the three best scores (fp32): sampler 0 entries, sampler 1 blocks; greedy rows: ty[0] = largest logit
   int tb[3];       // ... and their vocabulary / block indices, -1 = none
 };
@@ -123,23 +142,41 @@ static_assert(kPieceWords * 8 <= kPieceBytes, "piece size");
 struct WarpPartial {
   float M, Z, W;
   float zf;
+  float zmax;
   int err;
   float ty[3];
   int tb[3];
 };
 
+// What a ring slot holds; written by the warp's lane 0 when it starts the copy into the slot (tau arrives with
+// the data: a 4-byte asynchronous copy that completes on the slot's barrier).
+struct __align__(16) SliceMeta {
+  long long row;
+  int s_lo;      // first entry of the slice within its row
+  int n;         // entries of the slice (0: the warp holds nothing of this row piece, or the closing record)
+  uint32_t flags;
+  float tau;
+  uint32_t pad[2];
+};
+static_assert(sizeof(SliceMeta) == 32, "slot record");
+
 struct Smem {
-  u64 full[kStages], empty[kStages];  // ring barriers
+  u64 full[kStreamWarps][kStages];    // per warp and ring slot: the slot's data (and its tau) have landed
+  u64 empty[kStreamWarps][kStages];   // ... the warp is done with the slot
   u64 wfull[kSlots], wfree[kSlots];   // consumer warps -> finishing warp
-  u64 best64;                         // (segment number << 32 | encoded best score) of sampler 0
+  u64 best64;                         // (piece number << 32 | encoded best score) of sampler 0
+  SliceMeta meta[kStreamWarps][kStages];
   WarpPartial wpart[kSlots][kStreamWarps];
   int timeout;                        // set when a bounded wait ran out
+  unsigned long long deadline_ns;     // a wait that is still unsatisfied this long after it began gives up
+  int32_t *status;                    // the caller's status word (may be null)
+  uint32_t rk[20];                    // Philox round keys (a copy of the launch parameter: shared memory serves indexed reads best)
 };
 
 struct RowInfo {
   float tau, c;
   bool masked;   // masked out: the row's logits are not read and nothing is computed
-  bool invalid;  // temperature not usable: the logits still pass through the ring, unused
+  bool invalid;  // temperature not usable: the row's logits are not read either
   bool greedy;
 };
 
@@ -148,24 +185,13 @@ struct Seg {
   int e_lo, e_hi;  // entries [e_lo, e_hi) of the row
   bool whole;      // the CTA holds the whole row
   bool starts;     // holds the row's first tile
-  bool first;      // first segment of this CTA
+  bool slot0;      // cut piece that holds the CTA's first tile (workspace slot 0), else slot 1
   int k0, k1;      // CTAs holding the first / last tile of the row (cut rows only)
-};
-
-// Running sums of a consumer thread, two fp32 lanes per register pair.
-struct Acc {
-  float R, nRc;      // reference logit and -R*c; R = -inf, nRc = kNoRef: no reference yet
-  f2 Z2, W2;         // Z = sum of both halves of Z2, W likewise
-};
-// The same state as plain scalars (careful form).
-struct AccS {
-  float R, nRc, Z, W;
 };
 
 // Sampler 0: what a thread knows about the leaders of its row piece.  Scores are fp32 values of
 // y_i = z_i/tau + g_i, each within score_slack(y) of the exact value; the three best are kept so that
-// the finishing warp can tell whether fp32 separates the winner from the rest.  Greedy rows use
-// y[0] / b[0] for the largest logit and its index.
+// the finishing warp can tell whether fp32 separates the winner from the rest.
 struct Best {
   float y[3];
   int b[3];     // vocabulary indices, -1 = none; order: larger score first, equal scores by lower index
@@ -197,19 +223,24 @@ __device__ __forceinline__ f2 pack2f(float lo, float hi) { return make_float2(lo
 __device__ __forceinline__ float sum2(f2 v) { return v.x + v.y; }
 __device__ __forceinline__ f2 fma2(f2 a, f2 b, f2 c) { return __ffma2_rn(a, b, c); }
 __device__ __forceinline__ f2 add2(f2 a, f2 b) { return __fadd2_rn(a, b); }
-__device__ __forceinline__ f2 mul2(f2 a, f2 b) { return __fmul2_rn(a, b); }
-// max that keeps NaN (a NaN logit must reach the sums)
-__device__ __forceinline__ uint32_t floor_bf16x2(uint32_t w) {
-  uint32_t d;
-  asm("max.NaN.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(w), "r"(kFloorBf16x2));
-  return d;
-}
-__device__ __forceinline__ uint32_t floor_f32(uint32_t w) {
-  float d;
-  asm("max.NaN.f32 %0, %1, %2;" : "=f"(d) : "f"(__uint_as_float(w)), "f"(kFloorF32));
-  return __float_as_uint(d);
-}
 __device__ __forceinline__ uint32_t smem_addr(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ uint4 lds128(uint32_t addr) {
+  uint4 v;
+  asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+  return v;
+}
+template <int DT>
+__device__ __forceinline__ float lds_elem(uint32_t addr) {
+  if (DT == 0) {
+    float v;
+    asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(addr));
+    return v;
+  }
+  unsigned short h;
+  asm volatile("ld.shared.u16 %0, [%1];" : "=h"(h) : "r"(addr));
+  return __uint_as_float((uint32_t)h << 16);
+}
 
 __device__ __forceinline__ void mbar_init(u64 *b, int count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(b)), "r"(count) : "memory");
@@ -217,10 +248,11 @@ __device__ __forceinline__ void mbar_init(u64 *b, int count) {
 __device__ __forceinline__ void mbar_arrive(u64 *b) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(b)) : "memory");
 }
-__device__ __forceinline__ void mbar_arrive_expect_tx(u64 *b, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(b)), "r"(bytes) : "memory");
+__device__ __forceinline__ void mbar_expect_tx(u64 *b, uint32_t bytes) {
+  asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(b)), "r"(bytes) : "memory");
 }
-// One poll (the hardware may park the thread for a short, implementation-defined time).
+// One poll (the hardware may park the thread for a short, implementation-defined time; a loop of these
+// needs no sleep of its own, and a warp that has slept with nanosleep runs slowly for a while afterwards).
 __device__ __forceinline__ bool mbar_try_wait(u64 *b, uint32_t parity) {
   uint32_t ok;
   asm volatile(
@@ -230,30 +262,66 @@ __device__ __forceinline__ bool mbar_try_wait(u64 *b, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-// Bounded wait.  After any wait of the CTA has run out, no wait blocks any more.
-// sleep_ns > 0 parks the thread between polls (roles that mostly wait must not eat issue slots).
-__device__ __noinline__ void mbar_wait_slow(u64 *b, uint32_t parity, Smem &sm, unsigned sleep_ns) {
-  for (uint32_t it = 0; it < kSpinLimit; ++it) {
-    if (mbar_try_wait(b, parity)) return;
-    if (*reinterpret_cast<volatile int *>(&sm.timeout)) return;
-    if (sleep_ns) __nanosleep(sleep_ns);
-  }
+__device__ __forceinline__ unsigned long long global_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __forceinline__ bool timed_out(const Smem &sm) { return *reinterpret_cast<const volatile int *>(&sm.timeout) != 0; }
+// A wait has run out: from now on no wait of the CTA blocks, and the caller's status word says so.
+__device__ __noinline__ void raise_timeout(Smem &sm) {
   *reinterpret_cast<volatile int *>(&sm.timeout) = 1;
+  if (sm.status != nullptr) atomicOr(sm.status, kStatusTimeout);
 }
-__device__ __forceinline__ void mbar_wait(u64 *b, uint32_t parity, Smem &sm, unsigned sleep_ns = 0) {
-  if (!mbar_try_wait(b, parity)) mbar_wait_slow(b, parity, sm, sleep_ns);
+// Bounded wait: true when the barrier phase has completed, false when the wait was given up (it took longer
+// than the CTA's limit, or another wait of the CTA has run out before: then no wait blocks any more).
+__device__ __noinline__ bool mbar_wait_slow(u64 *b, uint32_t parity, Smem &sm) {
+  const unsigned long long t0 = global_ns();
+  for (uint32_t it = 1;; ++it) {
+    if (mbar_try_wait(b, parity)) return true;
+    if (timed_out(sm)) return false;
+    if ((it & 63u) == 0u && global_ns() - t0 > sm.deadline_ns) break;
+  }
+  raise_timeout(sm);
+  return false;
 }
-// Whole-warp wait with a single polling lane (used by the finishing warp, which mostly waits).
-__device__ __forceinline__ void mbar_wait_warp(u64 *b, uint32_t parity, Smem &sm, int lane) {
-  if (lane == 0) mbar_wait(b, parity, sm, 100u);
-  __syncwarp();
+__device__ __forceinline__ bool mbar_wait(u64 *b, uint32_t parity, Smem &sm) {
+  return mbar_try_wait(b, parity) ? true : mbar_wait_slow(b, parity, sm);
 }
-__device__ __forceinline__ void bulk_copy_g2s(void *dst, const void *src, uint32_t bytes, u64 *bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
-                   smem_addr(dst)),
-               "l"(src), "r"(bytes), "r"(smem_addr(bar))
+// Whole-warp wait with a single polling lane.
+__device__ __forceinline__ bool mbar_wait_warp(u64 *b, uint32_t parity, Smem &sm, int lane) {
+  bool ok = true;
+  if (lane == 0) ok = mbar_wait(b, parity, sm);
+  return __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+}
+// Bulk asynchronous copy global -> this CTA's shared memory; completion is counted in bytes on `bar`.
+// The logits are read once: their lines are marked evict-first in L2, so that the stream does not push out what
+// is used again and again (the kernel's instructions, the workspace, temperatures) -- an L2 miss of any of
+// those waits behind the whole queue of the stream.
+__device__ __forceinline__ u64 l2_evict_first_policy() {
+  u64 pol;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
+__device__ __forceinline__ void bulk_copy_g2s(uint32_t dst, const void *src, uint32_t bytes, u64 *bar, u64 policy) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;" ::"r"(dst),
+               "l"(src), "r"(bytes), "r"(smem_addr(bar)), "l"(policy)
                : "memory");
 }
+
+// Bulk asynchronous copy this CTA's shared memory -> global, as a bulk group of the issuing thread.
+__device__ __forceinline__ void bulk_store_s2g(void *dst, uint32_t src, uint32_t bytes) {
+  asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(src), "r"(bytes) : "memory");
+  asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+// Returns when all but the N most recent bulk groups of the thread have read their source.
+template <int N>
+__device__ __forceinline__ void bulk_wait_read() {
+  asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+// Orders the thread's earlier shared-memory writes before later reads of the asynchronous proxy (bulk copies).
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 // ---------------------------------------------------------------------------------------------
 // Philox4x32-10 (Salmon et al., SC'11) with precomputed round keys.
@@ -296,7 +364,7 @@ __device__ __forceinline__ int enc_float(float f) {
 __device__ __forceinline__ float dec_float(int e) { return __int_as_float(e >= 0 ? e : (e ^ 0x7FFFFFFF)); }
 __device__ __forceinline__ int enc_neg_inf() { return enc_float(-CUDART_INF_F); }
 
-// CTA-wide best score of the segment: 64-bit word (segment number, order-preserving code).
+// CTA-wide best score of the row piece: 64-bit word (piece number, order-preserving code).
 __device__ __forceinline__ void post_best(Smem &sm, uint32_t seg, int enc) {
   atomicMax(&sm.best64, ((u64)seg << 32) | (uint32_t)(enc ^ 0x80000000));
 }
@@ -314,33 +382,20 @@ __device__ __forceinline__ float load_elem(const char *row, int64_t i) {
   return __uint_as_float((uint32_t)__ldg(reinterpret_cast<const unsigned short *>(row) + i) << 16);
 }
 
-// 16 logits from global memory, entries at or beyond `valid` read as -inf.  Returns the largest.
+// 16 consecutive logits of a stage in shared memory (plain order).
 template <int DT>
-__device__ __forceinline__ float load_group_guarded(const char *row, int64_t e0, int valid, float (&z)[16]) {
-  float gmax = -CUDART_INF_F;
-#pragma unroll
-  for (int k = 0; k < 16; ++k) {
-    z[k] = k < valid ? load_elem<DT>(row, e0 + k) : -CUDART_INF_F;
-    gmax = fmaxf(gmax, z[k]);
-  }
-  return gmax;
-}
-
-// 16 logits that lie contiguously in shared memory (plain order).
-template <int DT>
-__device__ __forceinline__ void load_group_smem(const unsigned char *src, float (&z)[16]) {
+__device__ __forceinline__ void load_group_smem(uint32_t addr, float (&z)[16]) {
   if (DT == 0) {
-    const float4 *p = reinterpret_cast<const float4 *>(src);
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
-      const float4 v = p[q];
-      z[4 * q] = v.x; z[4 * q + 1] = v.y; z[4 * q + 2] = v.z; z[4 * q + 3] = v.w;
+      const uint4 v = lds128(addr + 16 * q);
+      z[4 * q] = __uint_as_float(v.x); z[4 * q + 1] = __uint_as_float(v.y);
+      z[4 * q + 2] = __uint_as_float(v.z); z[4 * q + 3] = __uint_as_float(v.w);
     }
   } else {
-    const uint4 *p = reinterpret_cast<const uint4 *>(src);
 #pragma unroll
     for (int q = 0; q < 2; ++q) {
-      const uint4 v = p[q];
+      const uint4 v = lds128(addr + 16 * q);
       const uint32_t w[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
@@ -354,130 +409,277 @@ __device__ __forceinline__ void load_group_smem(const unsigned char *src, float 
 // ---------------------------------------------------------------------------------------------
 // Running sums
 // ---------------------------------------------------------------------------------------------
-constexpr float kNoRef = 1e30f;  // nRc of a state without reference: the first group always overflows into the careful form
-
+// Running sums of a consumer thread, two fp32 lanes per register pair.
+struct Acc {
+  float R, nRc;      // reference logit and -R*c; R = -inf, nRc = kNoRef: no reference yet
+  f2 Z2, W2;         // Z = sum of both halves of Z2, W likewise
+};
 __device__ __forceinline__ void acc_reset(Acc &a) {
   a.R = -CUDART_INF_F;
   a.nRc = kNoRef;
   a.Z2 = a.W2 = pack2f(0.f, 0.f);
 }
-__device__ __forceinline__ AccS to_scalar(const Acc &a) {
-  AccS s;
-  s.R = a.R;
-  s.nRc = a.nRc;
-  s.Z = sum2(a.Z2);
-  s.W = sum2(a.W2);
-  return s;
-}
-__device__ __forceinline__ void from_scalar(Acc &a, const AccS &s) {
-  a.R = s.R;
-  a.nRc = s.nRc;
-  a.Z2 = pack2f(s.Z, 0.f);
-  a.W2 = pack2f(s.W, 0.f);
+
+// A thread's 128 bytes of a stage: B = shared-memory address of the slice with (lane mod 8) << 4 or-ed in;
+// v[i] is 16-byte vector number i xor (lane mod 8) of the slice.
+__device__ __forceinline__ void load_slice(uint32_t B, uint4 (&v)[8]) {
+#pragma unroll
+  for (int i = 0; i < 8; ++i) v[i] = lds128(B ^ (uint32_t)(i << 4));
 }
 
-// Careful form for one group: accepts any values.  -inf entries carry no weight, NaN and +inf flag the
-// row.  The reference moves up to max(R, ref_floor, largest logit of the group).  Returns the group's
-// sum of 2^t under the reference the state has afterwards.
-__device__ __forceinline__ float careful_accumulate(AccS &a, const float (&z)[16], float c, float ref_floor, int &err) {
-  float gmax = ref_floor;
-#pragma unroll
-  for (int k = 0; k < 16; ++k) {
-    if (z[k] != z[k]) err |= kErrValue;
-    gmax = fmaxf(gmax, z[k]);
-  }
-  if (gmax == CUDART_INF_F) {
-    err |= kErrValue;
-    return 0.f;
-  }
-  if (gmax > a.R) {
-    const float nRc = -gmax * c;
-    if (!(fabsf(nRc) < CUDART_INF_F)) {  // the product left the fp32 range
-      err |= kErrValue;
-      return 0.f;
-    }
-    const float d = nRc - a.nRc;
-    const float f = a.R == -CUDART_INF_F ? 0.f : ex2f(d);
-    if (f == 0.f) {
-      a.Z = a.W = 0.f;
-    } else {
-      a.W = f * fmaf(d, a.Z, a.W);
-      a.Z *= f;
-    }
-    a.R = gmax;
-    a.nRc = nRc;
-  }
-  float g = 0.f;
-#pragma unroll
-  for (int k = 0; k < 16; ++k) {
-    if (z[k] > -CUDART_INF_F) {  // false for NaN as well
-      const float t = fmaf(z[k], c, a.nRc), e = ex2f(t);
-      g += e;
-      a.W = fmaf(e, t, a.W);
-    }
-  }
-  a.Z += g;
-  return g;
-}
-
-// Largest logit of one group held in raw 16-byte vectors (NaN entries are passed over).
+// Entries at or beyond nlane (counted in vocabulary order within the slice) become -inf.
 template <int DT>
-__device__ __forceinline__ float group_max(const uint4 *v) {
-  if (DT == 1) {
-    uint32_t m = v[0].x;
+__device__ __forceinline__ void mask_slice(uint4 (&v)[8], int nlane, int r8) {
 #pragma unroll
-    for (int q = 0; q < 2; ++q) {
-      const uint32_t w[4] = {v[q].x, v[q].y, v[q].z, v[q].w};
+  for (int i = 0; i < 8; ++i) {
+    uint32_t w[4] = {v[i].x, v[i].y, v[i].z, v[i].w};
+    if (DT == 1) {
+      const int rem = nlane - 8 * (i ^ r8);  // entries of this vector that are valid
 #pragma unroll
-      for (int j = 0; j < 4; ++j) asm("max.bf16x2 %0, %1, %2;" : "=r"(m) : "r"(m), "r"(w[j]));
+      for (int j = 0; j < 4; ++j) {
+        const uint32_t lo = 2 * j < rem ? (w[j] & 0xFFFFu) : 0xFF80u;
+        const uint32_t hi = 2 * j + 1 < rem ? (w[j] & 0xFFFF0000u) : 0xFF800000u;
+        w[j] = lo | hi;
+      }
+    } else {
+      const int rem = nlane - 4 * (i ^ r8);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) w[j] = j < rem ? w[j] : 0xFF800000u;
     }
-    return fmaxf(__uint_as_float(m << 16), __uint_as_float(m & 0xFFFF0000u));
+    v[i] = make_uint4(w[0], w[1], w[2], w[3]);
+  }
+}
+
+// Largest logit of a slice (NaN entries are passed over).
+template <int DT>
+__device__ __forceinline__ float slice_max(const uint4 (&v)[8]) {
+  if (DT == 1) {
+    uint32_t m0 = v[0].x, m1 = v[0].y;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      asm("max.bf16x2 %0, %1, %2;" : "=r"(m0) : "r"(m0), "r"(v[i].x));
+      asm("max.bf16x2 %0, %1, %2;" : "=r"(m1) : "r"(m1), "r"(v[i].y));
+      asm("max.bf16x2 %0, %1, %2;" : "=r"(m0) : "r"(m0), "r"(v[i].z));
+      asm("max.bf16x2 %0, %1, %2;" : "=r"(m1) : "r"(m1), "r"(v[i].w));
+    }
+    asm("max.bf16x2 %0, %1, %2;" : "=r"(m0) : "r"(m0), "r"(m1));
+    return fmaxf(__uint_as_float(m0 << 16), __uint_as_float(m0 & 0xFFFF0000u));
   } else {
     float m = -CUDART_INF_F;
 #pragma unroll
-    for (int q = 0; q < 4; ++q)
-      m = fmaxf(fmaxf(m, fmaxf(__uint_as_float(v[q].x), __uint_as_float(v[q].y))),
-                fmaxf(__uint_as_float(v[q].z), __uint_as_float(v[q].w)));
+    for (int i = 0; i < 8; ++i)
+      m = fmaxf(fmaxf(m, fmaxf(__uint_as_float(v[i].x), __uint_as_float(v[i].y))),
+                fmaxf(__uint_as_float(v[i].z), __uint_as_float(v[i].w)));
     return m;
   }
 }
 
-// Streaming form for one group held in raw 16-byte vectors (any order): returns the packed sum of 2^t t in Wg2,
-// returns the packed group sum of 2^t in Zg2 and its scalar value.
-template <int DT, int NV>
-__device__ __forceinline__ float hot_vectors(const uint4 *v, f2 c2, f2 nRc2, f2 &Wg2, f2 &Zg2) {
-  f2 Za = pack2f(0.f, 0.f), Zb = pack2f(0.f, 0.f), Wa2 = pack2f(0.f, 0.f), Wb2 = pack2f(0.f, 0.f);
+// Streaming form for a slice: the packed sums of 2^t and of 2^t t over its entries, t = z c + nRc; with
+// GROUPS also the sum of 2^t of every group of 16 entries: Zg[j] belongs to group j xor ((lane mod 8) /
+// vectors per group).  CLAMP: logits below -2^100 (also -inf) enter as -2^100, which gives them weight 0 and
+// keeps 2^t t finite; NaN stays NaN.
+template <int DT, bool GROUPS, bool CLAMP>
+__device__ __forceinline__ void slice_sums(const uint4 (&v)[8], f2 c2, f2 nRc2, f2 &Zt2, f2 &Wt2, float (&Zg)[Fmt<DT>::kG]) {
+  constexpr int kVG = Fmt<DT>::kVG;
+  f2 Wa = pack2f(0.f, 0.f), Wb = pack2f(0.f, 0.f);
+  f2 Zj[Fmt<DT>::kG];
 #pragma unroll
-  for (int q = 0; q < NV; ++q) {
-    const uint32_t w[4] = {v[q].x, v[q].y, v[q].z, v[q].w};
+  for (int j = 0; j < Fmt<DT>::kG; ++j) Zj[j] = pack2f(0.f, 0.f);
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const uint32_t w[4] = {v[i].x, v[i].y, v[i].z, v[i].w};
 #pragma unroll
     for (int j = 0; j < (DT == 1 ? 4 : 2); ++j) {
       f2 z2;
       if (DT == 1) {
-        const uint32_t x = floor_bf16x2(w[j]);
+        uint32_t x = w[j];
+        if (CLAMP) asm("max.NaN.bf16x2 %0, %1, %2;" : "=r"(x) : "r"(x), "r"(0xF180F180u));
         z2 = pack2f(__uint_as_float(x << 16), __uint_as_float(x & 0xFFFF0000u));
       } else {
-        z2 = pack2f(__uint_as_float(floor_f32(w[2 * j])), __uint_as_float(floor_f32(w[2 * j + 1])));
+        float a = __uint_as_float(w[2 * j]), b = __uint_as_float(w[2 * j + 1]);
+        if (CLAMP) {
+          asm("max.NaN.f32 %0, %1, %2;" : "=f"(a) : "f"(a), "f"(-1.2676506e30f));
+          asm("max.NaN.f32 %0, %1, %2;" : "=f"(b) : "f"(b), "f"(-1.2676506e30f));
+        }
+        z2 = pack2f(a, b);
       }
       const f2 t2 = fma2(z2, c2, nRc2);
       const f2 e2 = pack2f(ex2f(t2.x), ex2f(t2.y));
-      if (j & 1) {
-        Zb = add2(Zb, e2);
-        Wb2 = fma2(e2, t2, Wb2);
-      } else {
-        Za = add2(Za, e2);
-        Wa2 = fma2(e2, t2, Wa2);
+      Zj[i / kVG] = add2(Zj[i / kVG], e2);
+      if (j & 1) Wb = fma2(e2, t2, Wb); else Wa = fma2(e2, t2, Wa);
+    }
+  }
+  Wt2 = add2(Wa, Wb);
+  if (GROUPS) {
+#pragma unroll
+    for (int j = 0; j < Fmt<DT>::kG; ++j) Zg[j] = sum2(Zj[j]);
+  }
+  if (Fmt<DT>::kG == 4) {
+    Zt2 = add2(add2(Zj[0], Zj[1]), add2(Zj[2], Zj[3]));
+  } else {
+    Zt2 = add2(Zj[0], Zj[1]);
+  }
+}
+
+// The streaming form as a loop over the two halves of the slice: the same sums (without group sums) with a
+// loop body short enough for the instruction cache.  The thread's slice is read in the order
+// i xor (lane mod 8) as everywhere.  GAP: zmax becomes the largest logit of the slice (NaN passed over).
+constexpr int kPartVecs = 4;
+template <int DT, bool GAP>
+__device__ __forceinline__ void slice_sums_rolled(uint32_t B, f2 c2, f2 nRc2, f2 &Zt2, f2 &Wt2, float &zmax) {
+  f2 Za = pack2f(0.f, 0.f), Zb = pack2f(0.f, 0.f), Wa = pack2f(0.f, 0.f), Wb = pack2f(0.f, 0.f);
+  uint32_t m0 = DT == 1 ? 0xFF80FF80u : 0xFF800000u, m1 = m0;  // -inf
+#pragma unroll 1
+  for (int h = 0; h < 8 / kPartVecs; ++h) {
+    const uint32_t Bh = B ^ (uint32_t)(h * kPartVecs * 16);
+    uint4 v[kPartVecs];
+#pragma unroll
+    for (int i = 0; i < kPartVecs; ++i) v[i] = lds128(Bh ^ (uint32_t)(i << 4));
+#pragma unroll
+    for (int i = 0; i < kPartVecs; ++i) {
+      const uint32_t w[4] = {v[i].x, v[i].y, v[i].z, v[i].w};
+      if (GAP) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          uint32_t &m = (j & 1) ? m1 : m0;
+          if (DT == 1) {
+            asm("max.bf16x2 %0, %1, %2;" : "=r"(m) : "r"(m), "r"(w[j]));
+          } else {
+            m = __float_as_uint(fmaxf(__uint_as_float(m), __uint_as_float(w[j])));
+          }
+        }
+      }
+#pragma unroll
+      for (int j = 0; j < (DT == 1 ? 4 : 2); ++j) {
+        f2 z2;
+        if (DT == 1) {
+          z2 = pack2f(__uint_as_float(w[j] << 16), __uint_as_float(w[j] & 0xFFFF0000u));
+        } else {
+          z2 = pack2f(__uint_as_float(w[2 * j]), __uint_as_float(w[2 * j + 1]));
+        }
+        const f2 t2 = fma2(z2, c2, nRc2);
+        const f2 e2 = pack2f(ex2f(t2.x), ex2f(t2.y));
+        if (j & 1) { Zb = add2(Zb, e2); Wb = fma2(e2, t2, Wb); } else { Za = add2(Za, e2); Wa = fma2(e2, t2, Wa); }
       }
     }
   }
-  Zg2 = add2(Za, Zb);
-  Wg2 = add2(Wa2, Wb2);
-  return sum2(Zg2);
+  Zt2 = add2(Za, Zb);
+  Wt2 = add2(Wa, Wb);
+  if (GAP) {
+    if (DT == 1) {
+      asm("max.bf16x2 %0, %1, %2;" : "=r"(m0) : "r"(m0), "r"(m1));
+      zmax = fmaxf(__uint_as_float(m0 << 16), __uint_as_float(m0 & 0xFFFF0000u));
+    } else {
+      zmax = fmaxf(__uint_as_float(m0), __uint_as_float(m1));
+    }
+  }
 }
 
+// The careful form of a turn: for the first turn of a row piece, for a slice that lies only partly inside the
+// piece, and when the streaming form's check failed (stale reference, a -inf, a NaN, a +inf).  The warp moves
+// its reference up to the largest finite logit of the slice, rescales its state and takes the turn with
+// masked and clamped entries.  A NaN or +inf (or numbers outside the fp32 range) flags the row.
 template <int DT>
-__device__ __forceinline__ float hot_group(const uint4 *v, f2 c2, f2 nRc2, f2 &Wg2, f2 &Zg2) {
-  return hot_vectors<DT, Fmt<DT>::kVG>(v, c2, nRc2, Wg2, Zg2);
+struct CarefulIO {
+  Acc acc;
+  f2 Zt2, Wt2;
+  float Zg[Fmt<DT>::kG];
+  float zmax;  // out: the lane's largest finite logit of the slice (-inf when it has none)
+  int err;
+};
+// Inlined: a call would spill the streaming loop's state to local memory around it, and with the memory
+// system saturated by the copies every such access takes microseconds.
+template <int DT, bool GROUPS>
+__device__ __forceinline__ void turn_careful(CarefulIO<DT> &io, uint32_t B, int nlane, int r8, float c) {
+  Acc acc = io.acc;
+  int err = io.err;
+  f2 Zt2, Wt2;
+  float Zg[Fmt<DT>::kG];
+  uint4 v[8];
+  load_slice(B, v);
+  if (nlane < Fmt<DT>::kLaneE) mask_slice<DT>(v, nlane, r8);
+  float gmax = slice_max<DT>(v);
+  if (!(gmax < CUDART_INF_F)) gmax = -CUDART_INF_F;  // +inf is flagged by the sums below
+  const float R0 = dec_float(__reduce_max_sync(0xffffffffu, enc_float(gmax)));
+  if (R0 > acc.R) {
+    const float nRc = -R0 * c;
+    if (fabsf(nRc) < CUDART_INF_F) {
+      const float d = nRc - acc.nRc;
+      const float f = acc.R == -CUDART_INF_F ? 0.f : ex2f(d);
+      if (f == 0.f) {
+        acc.Z2 = acc.W2 = pack2f(0.f, 0.f);
+      } else {
+        const f2 ff = pack2f(f, f);
+        acc.W2 = __fmul2_rn(ff, fma2(pack2f(d, d), acc.Z2, acc.W2));
+        acc.Z2 = __fmul2_rn(ff, acc.Z2);
+      }
+      acc.R = R0; acc.nRc = nRc;
+    } else {
+      err |= kErrValue;  // the product left the fp32 range
+    }
+  }
+  // without any reference (nothing finite so far) the sums must come out as zero
+  const float nRc_use = acc.R == -CUDART_INF_F ? 0.f : acc.nRc;
+  slice_sums<DT, GROUPS, true>(v, pack2f(c, c), pack2f(nRc_use, nRc_use), Zt2, Wt2, Zg);
+  const float Zs = sum2(Zt2), Ws = sum2(Wt2);
+  const bool bad = !(Zs <= kTurnSumMax) || !(fabsf(Ws) <= kTurnWMax) || (acc.R == -CUDART_INF_F && Zs != 0.f);
+  if (__any_sync(0xffffffffu, bad)) {
+    err |= kErrValue;
+    Zt2 = Wt2 = pack2f(0.f, 0.f);
+#pragma unroll
+    for (int j = 0; j < Fmt<DT>::kG; ++j) Zg[j] = 0.f;
+  }
+  io.acc = acc; io.err = err; io.Zt2 = Zt2; io.Wt2 = Wt2; io.zmax = gmax;
+#pragma unroll
+  for (int j = 0; j < Fmt<DT>::kG; ++j) io.Zg[j] = GROUPS ? Zg[j] : 0.f;
+}
+
+// What the bulk copy of a slice did not bring: the last bytes of a row whose length is no multiple of 16 bytes, or
+// everything when the rows do not start on 16-byte boundaries.  The warp fetches it entry by entry.
+template <int DT>
+__device__ __noinline__ void patch_slice(const char *row, int s_lo, int n, bool bulk, uint32_t dst, int lane) {
+  constexpr int kEsize = Fmt<DT>::kEsize;
+  const int ncopied = bulk ? (int)((((uint32_t)n * kEsize) & ~15u) / kEsize) : 0;
+  for (int e = ncopied + lane; e < n; e += 32) {
+    if (DT == 0) {
+      const float v = __ldg(reinterpret_cast<const float *>(row) + s_lo + e);
+      asm volatile("st.shared.f32 [%0], %1;" ::"r"(dst + e * 4), "f"(v) : "memory");
+    } else {
+      const unsigned short v = __ldg(reinterpret_cast<const unsigned short *>(row) + s_lo + e);
+      asm volatile("st.shared.u16 [%0], %1;" ::"r"(dst + e * 2), "h"(v) : "memory");
+    }
+  }
+  fence_async_smem();  // the next bulk copy into the slot comes after these stores
+  __syncwarp();
+}
+
+// Greedy rows (tau = 0): largest logit, lowest index; NaN and +inf flag the row.
+struct GreedyIO {
+  float y;
+  int i, err;
+};
+template <int DT>
+__device__ __noinline__ void turn_greedy(GreedyIO &io, uint32_t B, int e_lane, int nlane, int r8) {
+  float ybest = io.y;
+  int ibest = io.i, err = io.err;
+  uint4 v[8];
+  load_slice(B, v);
+  mask_slice<DT>(v, nlane, r8);
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const uint32_t w[4] = {v[i].x, v[i].y, v[i].z, v[i].w};
+    const int e0 = e_lane + (i ^ r8) * (DT == 1 ? 8 : 4);
+#pragma unroll
+    for (int k = 0; k < (DT == 1 ? 8 : 4); ++k) {
+      const float z = DT == 1 ? __uint_as_float((k & 1) ? (w[k >> 1] & 0xFFFF0000u) : (w[k >> 1] << 16)) : __uint_as_float(w[k]);
+      if (z != z || z == CUDART_INF_F) err |= kErrValue;
+      if (z > -CUDART_INF_F && (ibest < 0 || z > ybest || (z == ybest && e0 + k < ibest))) {
+        ybest = z;
+        ibest = e0 + k;
+      }
+    }
+  }
+  io.y = ybest; io.i = ibest; io.err = err;
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -561,16 +763,12 @@ __device__ __forceinline__ void consider(const uint32_t *rk, uint32_t grow, uint
   }
 }
 
-__device__ __noinline__ void eval_element(const EvalCtx &x, int i, uint32_t cbyte, float zf, Best &b, Smem &sm) {
-  consider(x.rk, x.grow, x.ctr_lo, x.ctr_hi8, x.tau, __frcp_rn(x.tau), x.slack_k, x.seg, i, cbyte, zf, b, sm);
-}
-
-// A queue entry holds one group: 16 coarse bytes, then its 16 logits in vocabulary order.  Its header
-// word is the index of the group's first entry, with bit 0 set when the group passed the sum gate.
+// A queue entry holds the 16 logits of one group in vocabulary order.  Its header word is the index
+// of the group's first entry, with bit 0 set when the group passed the sum gate.
 template <int DT>
 __device__ __forceinline__ float entry_logit(const unsigned char *entry, int k) {
-  if (DT == 0) return *reinterpret_cast<const float *>(entry + 16 + 4 * k);
-  return __uint_as_float((uint32_t)(*reinterpret_cast<const unsigned short *>(entry + 16 + 2 * k)) << 16);
+  if (DT == 0) return *reinterpret_cast<const float *>(entry + 4 * k);
+  return __uint_as_float((uint32_t)(*reinterpret_cast<const unsigned short *>(entry + 2 * k)) << 16);
 }
 
 // Evaluates the warp's queued groups, one per lane and round.  Everything it needs comes in registers
@@ -586,9 +784,10 @@ __device__ __noinline__ void drain_queue(const uint32_t *rk, uint32_t grow, uint
   const int *hdrs = reinterpret_cast<const int *>(queue);
 #pragma unroll 1
   for (int e = lane; e < qn; e += 32) {
-    const unsigned char *entry = queue + kQueueHdrBytes + e * Fmt<DT>::kEntryBytes;
+    const unsigned char *entry = queue + kQueueCap * 4 + e * Fmt<DT>::kEntryBytes;
     const int hdr = hdrs[e];
-    const uint4 cw = *reinterpret_cast<const uint4 *>(entry);
+    const int g0 = hdr & ~15;
+    const uint4 cw = philox(rk, (uint32_t)g0 >> 4, grow, ctr_lo, ctr_hi8 | 0u);  // the group's coarse bytes
     // bit k of todo: entry k of the group needs a look (its coarse byte is 255, or its logit is above the gate)
     uint32_t todo = 0;
     {
@@ -606,33 +805,21 @@ __device__ __noinline__ void drain_queue(const uint32_t *rk, uint32_t grow, uint
     while (todo) {
       const int k = __ffs(todo) - 1;
       todo &= todo - 1;
-      consider(rk, grow, ctr_lo, ctr_hi8, tau, inv_tau, slack_k, seg, (hdr & ~15) + k, entry[k], entry_logit<DT>(entry, k), b,
-               sm);
+      const uint32_t cbyte = (pick_word(cw, k >> 2) >> (8 * (k & 3))) & 0xFFu;
+      consider(rk, grow, ctr_lo, ctr_hi8, tau, inv_tau, slack_k, seg, g0 + k, cbyte, entry_logit<DT>(entry, k), b, sm);
     }
   }
   __syncwarp();
   best_io = b;
 }
 
-// Direct evaluation of one group held as floats (paths that do not stream from the ring).
-__device__ __forceinline__ void eval_group_direct(const EvalCtx &x, const float (&z)[16], int e0, int valid, Best &b,
-                                                  Smem &sm) {
-  if (valid <= 0) return;
-  const uint4 cw = philox(x.rk, (uint32_t)e0 >> 4, x.grow, x.ctr_lo, x.ctr_hi8 | 0u);
-#pragma unroll 1
-  for (int k = 0; k < valid; ++k) {
-    const uint32_t cbyte = (pick_word(cw, k >> 2) >> (8 * (k & 3))) & 0xFFu;
-    if (cbyte == 255u || z[k] > b.zthr) eval_element(x, e0 + k, cbyte, z[k], b, sm);
-  }
-}
-
 // ---------------------------------------------------------------------------------------------
 // Sampler 1: one Gumbel per block of 256 consecutive entries, applied to the block's log-sum-exp.
 // All lanes of a warp keep the same reference, so that the lane sums of a block add up directly.
-// kLB neighbouring lanes hold one block per step; every lane parks one block sum per kLB steps and
-// then all lanes turn their parked block into a score Y_b = L_b + g_b (one Philox call and three
-// MUFU each) and keep the three best (fp32).  The finishing warp settles near-ties in fp64 and
-// draws the token inside the winning block by inverse CDF.
+// kLB neighbouring lanes hold one block per stage; lane j of such a group keeps the block of stage j
+// of every kLB stages, and then all lanes turn the block they keep into a score Y_b = L_b + g_b (one
+// Philox call and three MUFU each) and enter it in their list of three leaders (fp32).  The finishing
+// warp settles near-ties in fp64 and draws the token inside the winning block by inverse CDF.
 // ---------------------------------------------------------------------------------------------
 struct Top3 {
   float y[3];
@@ -657,21 +844,8 @@ __device__ __forceinline__ void top3_insert(Top3 &t, float y, int b) {
   }
 }
 
-struct BlockState {
-  Top3 top;
-  float ref;  // parked block: its lane sums were taken under this reference
-  int b;      // its block index, -1: none
-};
-__device__ __forceinline__ void block_state_reset(BlockState &bs) {
-  top3_reset(bs.top);
-  bs.ref = 0.f; bs.b = -1;
-}
-
-// fp32 Gumbel variate of block b: u = (x + 1/2) 2^-32, g = -ln(-ln u)
-__device__ __forceinline__ float block_gumbel_f32(const uint32_t *rk, uint32_t grow, uint32_t ctr_lo, uint32_t ctr_hi8,
-                                                  int b) {
-  const uint4 w = philox(rk, (uint32_t)b >> 2, grow, ctr_lo, ctr_hi8 | 2u);
-  const uint32_t xw = pick_word(w, b & 3);
+// fp32 Gumbel variate from a 32-bit word: u = (x + 1/2) 2^-32, g = -ln(-ln u)
+__device__ __forceinline__ float gumbel_from_word(uint32_t xw) {
   float a;  // -ln u
   if (xw >= 0xFE000000u) {
     const float d = ((float)(~xw) + 0.5f) * 0x1p-32f;  // 1 - u < 2^-7: series of -ln(1 - d)
@@ -682,233 +856,33 @@ __device__ __forceinline__ float block_gumbel_f32(const uint32_t *rk, uint32_t g
   return -lg2f(a) * kLn2f;
 }
 
-// fp32 score of a block: ln sum_i exp(s_i) + g_b, from S = sum 2^(z c + ref).  Out of line (scalars in,
-// scalar out) so that the streaming loop stays short and its state stays in registers.
-__device__ __noinline__ float block_score(const uint32_t *rk, uint32_t grow, uint32_t ctr_lo, uint32_t ctr_hi8, float S,
-                                          float ref, int b) {
-  return (lg2f(S) - ref) * kLn2f + block_gumbel_f32(rk, grow, ctr_lo, ctr_hi8, b);
-}
-
-// Adds up the parked blocks of the warp (lane j of each group of kLB lanes owns the block of step j of
-// the current round; its lane sums sit in the warp's scratch) and enters their scores in the lane's list.
+// Sampler 0, first stage of a row piece: a valid lower bound of the piece's best score from the coarse byte
+// of the largest entry of each lane's first group alone: u >= (c + 2^-33)/256  =>  g >= -ln(ln 256 - ln(c + 2^-33)).
 template <int DT>
-__device__ __forceinline__ void block_flush(const uint32_t *rk, uint32_t grow, uint32_t ctr_lo, uint32_t ctr_hi8,
-                                            BlockState &bs, const float *scratch, int lane) {
-  constexpr int kLB = Fmt<DT>::kLB;
-  __syncwarp();
-  // row j of the scratch is rotated by 8 j columns, which spreads the lanes' reads over the banks
-  const int j = lane & (kLB - 1), col0 = (lane & ~(kLB - 1)) + 8 * j;
-  float S = 0.f;
-#pragma unroll
-  for (int i = 0; i < kLB / 4; ++i) {
-    const float4 v = *reinterpret_cast<const float4 *>(scratch + j * 32 + ((col0 + 4 * i) & 31));
-    S += (v.x + v.y) + (v.z + v.w);
-  }
-  __syncwarp();  // the scratch is written again in the next step
-  if (bs.b >= 0 && S > 0.f) top3_insert(bs.top, block_score(rk, grow, ctr_lo, ctr_hi8, S, bs.ref, bs.b), bs.b);
-  bs.b = -1;
-}
-
-// Step `it` of a warp in its row piece: every lane brings the sum of 2^t over its entries of this step
-// (all lanes under the reference nRc), which lie in block `b`; kLB neighbouring lanes share a block.
-// The lane sums go to the warp's scratch in shared memory and are added up only every kLB steps: one
-// read instead of a chain of shuffles at the end of every step.
-template <int DT>
-__device__ __forceinline__ void block_step(float zlane, int b, float nRc, const uint32_t *rk, uint32_t grow,
-                                           uint32_t ctr_lo, uint32_t ctr_hi8, BlockState &bs, float *scratch,
-                                           int lane, int it) {
-  constexpr int kLB = Fmt<DT>::kLB;
-  const int j = it & (kLB - 1);
-  scratch[j * 32 + ((lane + 8 * j) & 31)] = zlane;
-  if (j == (lane & (kLB - 1))) {
-    bs.ref = nRc;
-    bs.b = b;
-  }
-  if (j == kLB - 1) block_flush<DT>(rk, grow, ctr_lo, ctr_hi8, bs, scratch, lane);
-}
-
-// ---------------------------------------------------------------------------------------------
-// Out-of-line forms of one consumer step
-// ---------------------------------------------------------------------------------------------
-struct StepIO {
-  Acc acc;
-  float Zg[2];   // per group of the thread (vocabulary order): sum of 2^t under the final reference
-  float Zextra;  // a sum formed before this call, to be carried to the final reference
-  int err;
-};
-
-// Redo of the thread's groups of one stage in the careful form (a group sum left the safe range).
-// `have` bit g: group g of the thread is part of the row piece.  UNIFORM: all lanes of the warp are
-// here and must end with one common reference.
-template <int DT, bool UNIFORM>
-__device__ __noinline__ void redo_step(StepIO &io, const unsigned char *lane_data, int have, float c) {
-  constexpr int kG = Fmt<DT>::kG;
-  AccS a = to_scalar(io.acc);
-  const float nRc_old = a.nRc;
-  float z[kG][16];
-  float gm = -CUDART_INF_F;
-#pragma unroll
-  for (int g = 0; g < kG; ++g) {
-    if (have & (1 << g)) {
-      load_group_smem<DT>(lane_data + g * kGroup * Fmt<DT>::kEsize, z[g]);
-#pragma unroll
-      for (int k = 0; k < 16; ++k) gm = fmaxf(gm, z[g][k]);
-    } else {
-#pragma unroll
-      for (int k = 0; k < 16; ++k) z[g][k] = -CUDART_INF_F;
-    }
-  }
-  float ref_floor = -CUDART_INF_F;
-  if (UNIFORM) {
-    if (gm == CUDART_INF_F) gm = -CUDART_INF_F;  // flagged below; must not become the reference
-    ref_floor = dec_float(__reduce_max_sync(0xffffffffu, enc_float(gm)));
-  }
-  // settle the reference first, so that all group sums of this call refer to the same one
-  float top = ref_floor;
-#pragma unroll
-  for (int g = 0; g < kG; ++g)
-#pragma unroll
-    for (int k = 0; k < 16; ++k) top = fmaxf(top, z[g][k]);
-  if (top == CUDART_INF_F) top = ref_floor;
-#pragma unroll
-  for (int g = 0; g < kG; ++g) io.Zg[g] = careful_accumulate(a, z[g], c, top, io.err);
-  if (a.nRc != nRc_old) io.Zextra = nRc_old == kNoRef ? 0.f : io.Zextra * ex2f(a.nRc - nRc_old);
-  from_scalar(io.acc, a);
-}
-
-struct SlowIO {
-  Acc acc;
-  Best best;
-  float zsum;  // sum of 2^t over the entries handled by this call, under the final reference
-  int err;
-};
-
-// Up to kG groups of the thread read from global memory with guards: entries [e0, e_hi) of the row, at
-// most kLaneE of them.  Used for the last, partial group of a row, for rows that cannot use the ring
-// and for whatever else does not fit the streaming form.  SAMPLER 0 evaluates candidates directly.
-template <int DT, int SAMPLER, bool UNIFORM>
-__device__ __noinline__ void slow_groups(SlowIO &io, const EvalCtx &x, int e0, int e_hi, float c, Smem &sm) {
-  constexpr int kG = Fmt<DT>::kG;
-  AccS a = to_scalar(io.acc);
-  float z[kG][16];
-  int valid[kG];
-  float gm = -CUDART_INF_F;
-#pragma unroll
-  for (int g = 0; g < kG; ++g) {
-    const int g0 = e0 + g * kGroup;
-    valid[g] = e_hi - g0 < 0 ? 0 : (e_hi - g0 > kGroup ? kGroup : e_hi - g0);
-    if (valid[g] > 0) {
-      gm = fmaxf(gm, load_group_guarded<DT>(x.row, g0, valid[g], z[g]));
-    } else {
-#pragma unroll
-      for (int k = 0; k < 16; ++k) z[g][k] = -CUDART_INF_F;
-    }
-  }
-  float top = gm;
-  if (UNIFORM) {
-    if (gm == CUDART_INF_F) gm = -CUDART_INF_F;
-    top = dec_float(__reduce_max_sync(0xffffffffu, enc_float(gm)));
-  }
-  if (top == CUDART_INF_F) top = -CUDART_INF_F;
-  float zs = 0.f;
-#pragma unroll
-  for (int g = 0; g < kG; ++g) {
-    if (valid[g] > 0 || UNIFORM) zs += careful_accumulate(a, z[g], c, top, io.err);
-    if (SAMPLER == 0) eval_group_direct(x, z[g], e0 + g * kGroup, valid[g], io.best, sm);
-  }
-  io.zsum = zs;
-  from_scalar(io.acc, a);
-}
-
-// Greedy rows (tau = 0): largest logit, lowest index; NaN and +inf flag the row.  Full groups below
-// `lim` are read from the thread's 64 bytes of the pipeline stage (when there is one), the rest from
-// global memory with guards.
-template <int DT>
-__device__ __noinline__ void greedy_groups(SlowIO &io, const char *row, const unsigned char *lane_data, int e0, int lim,
-                                           int e_hi) {
-  constexpr int kG = Fmt<DT>::kG;
-#pragma unroll 1
-  for (int g = 0; g < kG; ++g) {
-    const int g0 = e0 + g * kGroup;
-    const int valid = e_hi - g0 < 0 ? 0 : (e_hi - g0 > kGroup ? kGroup : e_hi - g0);
-    if (valid <= 0) continue;
-    float z[16];
-    float gmax = -CUDART_INF_F;
-    if (lane_data != nullptr && g0 + kGroup <= lim) {
-      load_group_smem<DT>(lane_data + g * kGroup * Fmt<DT>::kEsize, z);
-#pragma unroll
-      for (int k = 0; k < 16; ++k) gmax = fmaxf(gmax, z[k]);
-    } else {
-      gmax = load_group_guarded<DT>(row, g0, valid, z);
-    }
-    int kk = -1;
-#pragma unroll
-    for (int k = 15; k >= 0; --k) {
-      if (z[k] != z[k] || z[k] == CUDART_INF_F) io.err |= kErrValue;
-      if (z[k] == gmax) kk = k;
-    }
-    if (kk >= 0 && gmax > -CUDART_INF_F && (io.best.b[0] < 0 || gmax > io.best.y[0])) {
-      io.best.y[0] = gmax;
-      io.best.b[0] = g0 + kk;
-    }
-  }
-}
-
-// The reference part of seed_piece alone, in line (no per-entry work): the largest finite logit among the
-// first groups of the warp's lanes, -inf if there is none.
-template <int DT>
-__device__ __forceinline__ float seed_reference(const unsigned char *lane_data, int e_lane, int lim) {
-  float gmax = -CUDART_INF_F;
-  if (e_lane + kGroup <= lim) {
-    uint4 v[Fmt<DT>::kVG];
-#pragma unroll
-    for (int i = 0; i < Fmt<DT>::kVG; ++i) v[i] = reinterpret_cast<const uint4 *>(lane_data)[i];
-    gmax = group_max<DT>(v);
-  }
-  if (!(gmax < CUDART_INF_F)) gmax = -CUDART_INF_F;
-  return dec_float(__reduce_max_sync(0xffffffffu, enc_float(gmax)));
-}
-
-struct SeedIO {
-  float R0;  // warp-wide reference, -inf = none found
-  Best best;
-};
-
-// First stage of a row piece: a common reference for the warp from each lane's first group, and for
-// sampler 0 a valid lower bound of the piece's best score from the coarse byte of each lane's largest
-// entry alone: u >= (c + 2^-33)/256  =>  g >= -ln(ln 256 - ln(c + 2^-33)).
-template <int DT, int SAMPLER>
-__device__ __noinline__ void seed_piece(SeedIO &io, const EvalCtx &x, const unsigned char *lane_data, int e_lane,
-                                        int lim, Smem &sm) {
-  const bool have = e_lane + kGroup <= lim;
+__device__ __noinline__ void seed_gate(Best &best, const EvalCtx &x, uint32_t lane_addr, int e_lane, Smem &sm) {
   float z[16];
+  load_group_smem<DT>(lane_addr, z);
   float gmax = -CUDART_INF_F;
-  if (have) {
-    load_group_smem<DT>(lane_data, z);
 #pragma unroll
-    for (int k = 0; k < 16; ++k) gmax = fmaxf(gmax, z[k]);
-  }
-  const bool usable = have && gmax > -CUDART_INF_F && gmax < CUDART_INF_F;
-  io.R0 = dec_float(__reduce_max_sync(0xffffffffu, enc_float(usable ? gmax : -CUDART_INF_F)));
-  if (SAMPLER == 0) {
-    float ylo = -CUDART_INF_F;
-    if (usable) {
-      const uint4 cb = philox(x.rk, (uint32_t)e_lane >> 4, x.grow, x.ctr_lo, x.ctr_hi8 | 0u);
-      uint32_t cbyte = 0;
+  for (int k = 0; k < 16; ++k) gmax = fmaxf(gmax, z[k]);
+  const bool usable = gmax > -CUDART_INF_F && gmax < CUDART_INF_F;
+  float ylo = -CUDART_INF_F;
+  if (usable) {
+    const uint4 cb = philox(x.rk, (uint32_t)e_lane >> 4, x.grow, x.ctr_lo, x.ctr_hi8 | 0u);
+    uint32_t cbyte = 0;
 #pragma unroll
-      for (int k = 15; k >= 0; --k)
-        if (z[k] == gmax) cbyte = (pick_word(cb, k >> 2) >> (8 * (k & 3))) & 0xFFu;
-      const float neg_ln_u = (8.0f - lg2f((float)cbyte + 0x1p-33f)) * kLn2f;
-      const float glo = -lg2f(neg_ln_u) * kLn2f;
-      const float sf = gmax / x.tau;
-      ylo = sf - fabsf(sf) * 8e-6f + glo - 4e-3f;  // also five score slacks below the entry's score
-    }
-    int enc = __reduce_max_sync(0xffffffffu, enc_float(ylo));
-    if ((threadIdx.x & 31) == 0 && enc > enc_neg_inf()) post_best(sm, x.seg, enc);
-    const int cta = read_best(sm, x.seg);
-    enc = enc > cta ? enc : cta;
-    if (enc > io.best.enc) set_gate(io.best, enc, x.tau);
+    for (int k = 15; k >= 0; --k)
+      if (z[k] == gmax) cbyte = (pick_word(cb, k >> 2) >> (8 * (k & 3))) & 0xFFu;
+    const float neg_ln_u = (8.0f - lg2f((float)cbyte + 0x1p-33f)) * kLn2f;
+    const float glo = -lg2f(neg_ln_u) * kLn2f;
+    const float sf = gmax / x.tau;
+    ylo = sf - fabsf(sf) * 8e-6f + glo - 4e-3f;  // also five score slacks below the entry's score
   }
+  int enc = __reduce_max_sync(0xffffffffu, enc_float(ylo));
+  if ((threadIdx.x & 31) == 0 && enc > enc_neg_inf()) post_best(sm, x.seg, enc);
+  const int cta = read_best(sm, x.seg);
+  enc = enc > cta ? enc : cta;
+  if (enc > best.enc) set_gate(best, enc, x.tau);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -956,12 +930,44 @@ __device__ __forceinline__ bool piece_load(const u64 *src, u64 call_id, Piece &p
   memcpy(&pc, w, sizeof(Piece));
   return ok;
 }
+// Makes a piece unreadable for every call id: word j gets the complement of this call's tag.
+__device__ __forceinline__ void piece_wipe(u64 *dst, u64 call_id) {
+#pragma unroll
+  for (int j = 0; j < kPieceWords; ++j) {
+    const u64 v = (u64)(~piece_tag(call_id, j)) << 32;
+    asm volatile("st.relaxed.gpu.global.b64 [%0], %1;" ::"l"(dst + j), "l"(v) : "memory");
+  }
+}
+
+// Merges the lists of leaders held by the 32 lanes of a warp (sampler 0 entries, sampler 1 blocks, greedy
+// maxima); every lane ends with the result, zf follows top.b[0].  Three rounds of "take the best head":
+// larger score first, equal scores by lower index.
+__device__ __forceinline__ void warp_merge_top(Top3 &top, float &zf) {
+  constexpr unsigned kAll = 0xffffffffu;
+  Top3 out;
+  top3_reset(out);
+  int pos = 0;
+#pragma unroll
+  for (int r = 0; r < 3; ++r) {
+    const float hy = pos == 0 ? top.y[0] : (pos == 1 ? top.y[1] : top.y[2]);
+    const int hb = pos >= 3 ? -1 : (pos == 0 ? top.b[0] : (pos == 1 ? top.b[1] : top.b[2]));
+    const int e = hb >= 0 ? enc_float(hy) : INT_MIN;
+    const int emax = __reduce_max_sync(kAll, e);
+    if (emax != INT_MIN) {
+      const bool c2 = hb >= 0 && e == emax;
+      const int bmin = __reduce_min_sync(kAll, c2 ? hb : INT_MAX);
+      out.y[r] = dec_float(emax);
+      out.b[r] = bmin;
+      const bool mine = c2 && hb == bmin;
+      if (r == 0) zf = __shfl_sync(kAll, zf, __ffs(__ballot_sync(kAll, mine)) - 1);
+      if (mine) ++pos;
+    }
+  }
+  top = out;
+}
 
 // Merges the partial states held by the 32 lanes of a warp; every lane ends with the result.  A lane
-// without weight (Z = 0) or with an empty list takes no part.  Written with warp-wide reductions so
-// that the chain of dependent instructions stays short: this runs at the end of every row piece, when
-// nothing else can hide it.  The order of all sums is fixed by lane numbers.  with_top: the lists of
-// leaders (sampler 0 entries, sampler 1 blocks, greedy maxima) are merged too; pc.zf follows top.b[0].
+// without weight (Z = 0) takes no part.  The order of all sums is fixed by lane numbers.
 __device__ __forceinline__ void warp_merge(Piece &pc, Top3 &top, bool with_top) {
   constexpr unsigned kAll = 0xffffffffu;
   // softmax sums: move every lane to the largest reference, then add
@@ -983,29 +989,8 @@ __device__ __forceinline__ void warp_merge(Piece &pc, Top3 &top, bool with_top) 
   }
   pc.M = Mw; pc.Z = Zs; pc.W = Ws;
   pc.err = __reduce_or_sync(kAll, pc.err);
-  if (with_top) {
-    // three rounds of "take the best head": larger score first, equal scores by lower index
-    Top3 out;
-    top3_reset(out);
-    int pos = 0;
-#pragma unroll
-    for (int r = 0; r < 3; ++r) {
-      const float hy = pos == 0 ? top.y[0] : (pos == 1 ? top.y[1] : top.y[2]);
-      const int hb = pos >= 3 ? -1 : (pos == 0 ? top.b[0] : (pos == 1 ? top.b[1] : top.b[2]));
-      const int e = hb >= 0 ? enc_float(hy) : INT_MIN;
-      const int emax = __reduce_max_sync(kAll, e);
-      if (emax != INT_MIN) {
-        const bool c2 = hb >= 0 && e == emax;
-        const int bmin = __reduce_min_sync(kAll, c2 ? hb : INT_MAX);
-        out.y[r] = dec_float(emax);
-        out.b[r] = bmin;
-        const bool mine = c2 && hb == bmin;
-        if (r == 0) pc.zf = __shfl_sync(kAll, pc.zf, __ffs(__ballot_sync(kAll, mine)) - 1);
-        if (mine) ++pos;
-      }
-    }
-    top = out;
-  }
+  pc.zmax = dec_float(__reduce_max_sync(kAll, enc_float(pc.zmax)));
+  if (with_top) warp_merge_top(top, pc.zf);
 }
 
 // Largest y over the lanes, then lowest index (lanes with idx < 0 take no part); all lanes get the winner.
@@ -1045,87 +1030,96 @@ __device__ __forceinline__ int cta_of_tile(const RowsParams &p, int64_t t) {
   return (int)(t < big ? quot(p, t, p.tiles_q + 1) : p.tiles_r + quot(p, t - big, p.tiles_q));
 }
 
-// Hands out the CTA's row pieces one after the other.  The only state is a count of what has been
-// handed out; everything else is recomputed from the launch parameters (registers are scarce here).
+// Hands out the CTA's row pieces: first the piece that starts inside a row (if the run starts so), then
+// the piece that ends inside a row, then the whole rows in order.  All divisions happen in the constructor.
 struct Walker {
-  int rel;  // tiles of the CTA's run handed out so far (interleaved: rows handed out)
-  __device__ Walker() : rel(0) {}
-  __device__ static int64_t run_length(const RowsParams &p) { return p.tiles_q + ((int64_t)blockIdx.x < p.tiles_r ? 1 : 0); }
-  // Row of the first piece, -1 when the CTA has nothing to do.
-  __device__ static int64_t first_row(const RowsParams &p) {
-    if (p.interleaved) return (int64_t)blockIdx.x < p.rows ? (int64_t)blockIdx.x : -1;
-    return run_length(p) > 0 ? quot(p, first_tile_of(p, blockIdx.x), p.tiles_per_row) : -1;
+  int64_t row0;     // row of the run's first tile (interleaved: the CTA's first row)
+  int n;            // pieces of the run in vocabulary order (interleaved: rows of the CTA)
+  int tin0, tend;   // first tile of the run within row0; end tile of the run within its last row (1..tiles_per_row)
+  int k;            // pieces handed out so far
+  bool first_cut, last_cut;
+  __device__ explicit Walker(const RowsParams &p) : row0(0), n(0), tin0(0), tend(0), k(0), first_cut(false), last_cut(false) {
+    if (p.interleaved) {
+      row0 = blockIdx.x;
+      n = (int64_t)blockIdx.x < p.rows ? (int)((p.rows - 1 - blockIdx.x) / gridDim.x) + 1 : 0;
+      return;
+    }
+    const int64_t len = p.tiles_q + ((int64_t)blockIdx.x < p.tiles_r ? 1 : 0);
+    if (len <= 0) return;
+    const int64_t t0 = first_tile_of(p, blockIdx.x);
+    row0 = quot(p, t0, p.tiles_per_row);
+    tin0 = (int)(t0 - row0 * p.tiles_per_row);
+    const int64_t row_last = quot(p, t0 + len - 1, p.tiles_per_row);
+    tend = (int)(t0 + len - row_last * p.tiles_per_row);
+    n = (int)(row_last - row0) + 1;
+    const int tpr = (int)p.tiles_per_row;
+    first_cut = tin0 > 0 || (n == 1 && tend < tpr);
+    last_cut = n > 1 && tend < tpr;
   }
-  // Row of the piece after `cur` (the piece handed out last), -1 when there is none.
-  __device__ int64_t row_after(const RowsParams &p, const Seg &cur) const {
-    if (p.interleaved) return cur.row + gridDim.x < p.rows ? cur.row + gridDim.x : -1;
-    return rel < run_length(p) ? cur.row + 1 : -1;
+  // Row of the piece number q of the hand-out order (q >= 0), -1 when there is none.
+  __device__ int64_t row_of(const RowsParams &p, int q) const {
+    if (q >= n) return -1;
+    if (p.interleaved) return row0 + (int64_t)q * gridDim.x;
+    return row0 + index_of(q);
+  }
+  __device__ int index_of(int q) const {  // hand-out number -> position in vocabulary order
+    const int nc = (first_cut ? 1 : 0) + (last_cut ? 1 : 0);
+    if (q == 0 && first_cut) return 0;
+    if (q == (first_cut ? 1 : 0) && last_cut) return n - 1;
+    return q - nc + (first_cut ? 1 : 0);
   }
   // with_range: also work out which CTAs hold the row's first and last tile (only the finishing warp asks)
+  template <int DT>
   __device__ bool next(const RowsParams &p, Seg &s, bool with_range) {
+    if (k >= n) return false;
+    s.k0 = s.k1 = 0;
     if (p.interleaved) {
-      const int64_t row = (int64_t)blockIdx.x + (int64_t)rel * gridDim.x;
-      if (row >= p.rows) return false;
-      s.row = row; s.e_lo = 0; s.e_hi = (int)p.V; s.whole = true; s.starts = true; s.first = rel == 0; s.k0 = s.k1 = 0;
-      ++rel;
+      s.row = row0 + (int64_t)k * gridDim.x;
+      s.e_lo = 0; s.e_hi = (int)p.V; s.whole = true; s.starts = true; s.slot0 = false;
+      ++k;
       return true;
     }
-    const int64_t len = run_length(p);
-    if (rel >= len) return false;
-    // only the CTA's first piece can start inside a row: every later one starts the row after `s.row`
-    // (s still holds the piece handed out before)
-    int64_t row, tin;
-    if (rel == 0) {
-      const int64_t t = first_tile_of(p, blockIdx.x);
-      row = quot(p, t, p.tiles_per_row);
-      tin = t - row * p.tiles_per_row;
-    } else {
-      row = s.row + 1;
-      tin = 0;
-    }
-    const int64_t n = p.tiles_per_row - tin < len - rel ? p.tiles_per_row - tin : len - rel;
-    const int64_t lo = tin * kTile, hi = (tin + n) * kTile;
-    s.row = row;
-    s.e_lo = (int)(lo < p.V ? lo : p.V);
-    s.e_hi = (int)(hi < p.V ? hi : p.V);
-    s.starts = tin == 0;
-    s.whole = tin == 0 && n == p.tiles_per_row;
-    s.first = rel == 0;
-    s.k0 = s.k1 = 0;
+    const int j = index_of(k);
+    const int tpr = (int)p.tiles_per_row;
+    const int lo = j == 0 ? tin0 : 0, hi = j == n - 1 ? tend : tpr;
+    const int64_t elo = (int64_t)lo * Fmt<DT>::kWarpE, ehi = (int64_t)hi * Fmt<DT>::kWarpE;
+    s.row = row0 + j;
+    s.e_lo = (int)elo;
+    s.e_hi = (int)(ehi < p.V ? ehi : p.V);
+    s.starts = lo == 0;
+    s.whole = lo == 0 && hi == tpr;
+    s.slot0 = j == 0;
     if (!s.whole && with_range) {
-      s.k0 = cta_of_tile(p, row * p.tiles_per_row);
-      s.k1 = cta_of_tile(p, (row + 1) * p.tiles_per_row - 1);
+      s.k0 = cta_of_tile(p, s.row * p.tiles_per_row);
+      s.k1 = cta_of_tile(p, (s.row + 1) * p.tiles_per_row - 1);
     }
-    rel += (int)n;
+    ++k;
     return true;
   }
 };
 
 // Walks the CTA's row pieces and loads temperature and mask of the piece after the current one, so
-// that nobody waits for them when that piece starts.  The copy-issuing thread passes with_tau = false:
-// it only needs the mask, and must not wait for anything before its first copy.
+// that nobody waits for them when that piece starts.
+template <int DT>
 struct SegIter {
   Walker wk;
   float tau_next;
   bool masked_next;
-  bool with_tau, with_range;
-  __device__ SegIter(const RowsParams &p, bool with_tau_, bool with_range_ = false)
-      : with_tau(with_tau_), with_range(with_range_) {
-    prefetch(p, Walker::first_row(p));
-  }
+  bool with_range;
+  __device__ SegIter(const RowsParams &p, bool with_range_) : wk(p), with_range(with_range_) { prefetch(p, wk.row_of(p, 0)); }
   __device__ void prefetch(const RowsParams &p, int64_t row) {
     tau_next = p.temp_scalar;
     masked_next = false;
     if (row >= 0) {
-      if (with_tau && p.temps) tau_next = __ldg(p.temps + row);
+      if (p.temps) tau_next = __ldg(p.temps + row);
       masked_next = p.mode != kModeSample && p.mask && __ldg(p.mask + row) == 0;
     }
   }
   __device__ bool next(const RowsParams &p, Seg &s, RowInfo &r) {
-    if (!wk.next(p, s, with_range)) return false;
+    if (!wk.template next<DT>(p, s, with_range)) return false;
     r.tau = tau_next;
     r.masked = masked_next;
-    prefetch(p, wk.row_after(p, s));
+    prefetch(p, wk.row_of(p, wk.k));
     r.greedy = p.mode == kModeSample && r.tau == 0.f;
     r.invalid = !r.masked && !r.greedy && !(r.tau > 0.f && r.tau < CUDART_INF_F);
     r.c = r.greedy || r.masked || r.invalid ? 0.f : __fdiv_rn(kLog2e, r.tau);
@@ -1141,24 +1135,32 @@ __device__ __forceinline__ const char *row_ptr(const RowsParams &p, int64_t row)
 // ---------------------------------------------------------------------------------------------
 // Row epilogue (one thread, fp64).  zt: logit of the token whose log-probability is wanted.
 // ---------------------------------------------------------------------------------------------
+// defer: the token of this row is drawn by block_sample_kernel, which gets the row's sums through the workspace
+// (x: reference in log2 units, y: sum of 2^t, z: non-zero = nothing to do, the row is finished or flagged).
 __device__ __forceinline__ void finish_row(const RowsParams &p, int64_t row, const RowInfo &ri, float Mf, float Zf,
-                                           float Wf, int idx, int err, bool have_zt, float zt, bool store) {
+                                           float Wf, float zmax, int idx, int err, bool have_zt, float zt, bool defer) {
   const double M = Mf, Z = Zf, W = Wf;
   const bool sample = p.mode == kModeSample;
   int tok = -1;
-  float logp = CUDART_NAN_F, ent = CUDART_NAN_F;
+  float logp = CUDART_NAN_F, ent = CUDART_NAN_F, gap = CUDART_NAN_F;
+  bool deferred = false;
   if (ri.greedy) {
-    if (err == 0 && idx >= 0) { tok = idx; logp = 0.f; ent = 0.f; }
+    if (err == 0 && idx >= 0) { tok = idx; logp = 0.f; ent = 0.f; gap = 0.f; }
   } else if (err == 0 && Z > 0.0) {
     const double lnZ = log(Z);
     ent = (float)(lnZ - kLn2 * (W / Z));
+    // sum p_i (s_max - s_i) with s = z/tau: the mean of s is (M + W/Z) ln2
+    gap = (float)(((double)zmax * (double)ri.c - M - W / Z) * kLn2);
     if (sample) tok = idx;
     if (have_zt) logp = (float)(((double)zt * (double)ri.c - M) * kLn2 - lnZ);
+    deferred = defer;
   }
-  if (!store) return;
+  if (defer) p.ws_rowstat[row] = make_float4(Mf, Zf, deferred ? 0.f : 1.f, 0.f);
+  if (p.out_ent) p.out_ent[row] = ent;
+  if (p.out_gap) p.out_gap[row] = gap;
+  if (deferred) return;
   if (sample) p.out_tok[row] = tok;
   if (p.out_logp) p.out_logp[row] = logp;
-  if (p.out_ent) p.out_ent[row] = ent;
 }
 
 __device__ __forceinline__ void write_skipped(const RowsParams &p, int64_t row, const RowInfo &ri) {
@@ -1167,6 +1169,15 @@ __device__ __forceinline__ void write_skipped(const RowsParams &p, int64_t row, 
   if (sample) p.out_tok[row] = -1;
   if (p.out_logp) p.out_logp[row] = v;
   if (p.out_ent) p.out_ent[row] = v;
+  if (p.out_gap) p.out_gap[row] = v;
+}
+// A row the CTA gives up on (a wait ran out).
+__device__ __forceinline__ void write_abandoned(const RowsParams &p, int64_t row, bool defer) {
+  if (p.mode == kModeSample) p.out_tok[row] = -1;
+  if (p.out_logp) p.out_logp[row] = CUDART_NAN_F;
+  if (p.out_ent) p.out_ent[row] = CUDART_NAN_F;
+  if (p.out_gap) p.out_gap[row] = CUDART_NAN_F;
+  if (defer) p.ws_rowstat[row] = make_float4(0.f, 0.f, 1.f, 0.f);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -1400,24 +1411,122 @@ __device__ __noinline__ int settle_exact(const EvalCtx &x, const Top3 &top, floa
 // ---------------------------------------------------------------------------------------------
 // The kernel
 // ---------------------------------------------------------------------------------------------
-template <int DT, int SAMPLER, bool RING>
+// 4-byte asynchronous copy global -> shared and an arrival on `bar` once the thread's earlier copies of this
+// kind have landed (the arrival counts as one of the barrier's expected arrivals).
+__device__ __forceinline__ void async_copy4(uint32_t dst, const void *src) {
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void async_arrive(u64 *bar) {
+  asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(smem_addr(bar)) : "memory");
+}
+
+// Keeps the ring of one consumer warp filled: lane w of the feeding warp does this for consumer warp w.  It
+// walks the CTA's row pieces; of every piece the consumer warp takes the slices
+// [e_lo + q * (entries per stage) + w * (entries per slice), + entries per slice) that start inside the
+// piece; a piece of which the warp holds nothing still gives one empty record, so that every warp hands
+// exactly one partial state per piece to the finishing warp.  Only whole 16-byte units are copied here (one
+// bulk copy per slice); what a row whose length is no multiple of 16 bytes leaves over, and rows that do not
+// start on 16-byte boundaries altogether, the consumer warp fetches itself.
+template <int DT>
+struct Feeder {
+  Walker wk;
+  int64_t row;
+  int s_next, e_hi, q_left;
+  bool first, done, stalled, masked_next;
+  u64 policy;
+  __device__ Feeder(const RowsParams &p) : wk(p), row(0), s_next(0), e_hi(0), q_left(0), first(false), done(false), stalled(false) {
+    policy = l2_evict_first_policy();
+    masked_next = false;
+    peek_mask(p, wk.row_of(p, 0));
+  }
+  __device__ void peek_mask(const RowsParams &p, int64_t r) {
+    masked_next = r >= 0 && p.mode != kModeSample && p.mask && __ldg(p.mask + r) == 0;
+  }
+  // Puts the next slice of consumer warp w (or the closing record) into its ring slot `slot`.
+  __device__ __forceinline__ void feed(const RowsParams &p, Smem &sm, uint32_t ring, int w, int slot) {
+    using F = Fmt<DT>;
+    uint32_t flags;
+    int n;
+    SliceMeta m;
+    m.pad[0] = m.pad[1] = 0;
+    u64 *const bar = &sm.full[w][slot];
+    if (q_left == 0) {
+      Seg s;
+      bool have;
+      for (;;) {
+        have = wk.template next<DT>(p, s, false);
+        if (!have) break;
+        const bool masked = masked_next;
+        peek_mask(p, wk.row_of(p, wk.k));
+        if (!masked) break;
+      }
+      if (!have) {
+        done = true;
+        m.row = 0; m.s_lo = 0; m.n = 0; m.flags = kFlagEnd; m.tau = 0.f;
+        sm.meta[w][slot] = m;
+        mbar_arrive(bar);
+        return;
+      }
+      row = s.row;
+      e_hi = s.e_hi;
+      s_next = s.e_lo + w * F::kWarpE;
+      q_left = s_next < e_hi ? (e_hi - s_next + F::kStageE - 1) / F::kStageE : 0;
+      first = true;
+    }
+    if (q_left == 0) {  // nothing of this piece lies in the warp's slices
+      flags = kFlagFirst | kFlagLast;
+      n = 0;
+    } else {
+      flags = (first ? kFlagFirst : 0u) | (q_left == 1 ? kFlagLast : 0u);
+      n = e_hi - s_next < F::kWarpE ? e_hi - s_next : F::kWarpE;
+    }
+    if (p.stall_tile >= 0 && n > 0 && row * p.tiles_per_row + s_next / F::kWarpE == p.stall_tile) {
+      done = stalled = true;  // test hook: this slot is never filled, the consumer's wait for it runs out
+      return;
+    }
+    m.row = row; m.s_lo = s_next; m.n = n; m.flags = flags; m.tau = p.temp_scalar;
+    sm.meta[w][slot] = m;
+    const uint32_t bytes = p.bulk ? ((uint32_t)n * F::kEsize) & ~15u : 0u;
+    if (bytes > 0) {
+      mbar_expect_tx(bar, bytes);
+      bulk_copy_g2s(ring + (uint32_t)slot * kWarpBytes, row_ptr<DT>(p, row) + (size_t)s_next * F::kEsize, bytes, bar, policy);
+    }
+    if (p.temps != nullptr) {
+      async_copy4(smem_addr(&sm.meta[w][slot].tau), p.temps + row);
+      async_arrive(bar);
+    } else {
+      mbar_arrive(bar);
+    }
+    if (q_left > 0) {
+      s_next += F::kStageE;
+      --q_left;
+    }
+    first = false;
+  }
+};
+
+// GAP: also track the largest logit of every row (for the mean logit gap).
+template <int DT, int SAMPLER, bool GAP>
 __global__ void __launch_bounds__(kThreads, 2) rows_kernel(const __grid_constant__ RowsParams p) {
-  extern __shared__ __align__(128) unsigned char dyn[];  // ring, then sampler 0: candidate queues, sampler 1: lane sums
+  extern __shared__ __align__(128) unsigned char dyn[];  // the warps' rings, then sampler 0: candidate queues
   __shared__ Smem sm;
   using F = Fmt<DT>;
   constexpr int kEsize = F::kEsize;
-  constexpr int kChunkE = F::kChunkE;
   constexpr int kLaneE = F::kLaneE;
   constexpr int kG = F::kG;
-  constexpr int kVG = F::kVG;
+  constexpr int kNS = RingStages<DT, SAMPLER>::value;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  unsigned char *const ring = dyn;
+  const uint32_t ring = smem_addr(dyn);
 
   if (tid == 0) {
-    for (int s = 0; s < kStages; ++s) { mbar_init(&sm.full[s], 1); mbar_init(&sm.empty[s], kStreamWarps); }
+    for (int w = 0; w < kStreamWarps; ++w)
+      for (int s = 0; s < kNS; ++s) { mbar_init(&sm.full[w][s], 1); mbar_init(&sm.empty[w][s], 1); }
     for (int s = 0; s < kSlots; ++s) { mbar_init(&sm.wfull[s], kStreamWarps); mbar_init(&sm.wfree[s], 1); }
     sm.best64 = 0ull;
     sm.timeout = 0;
+    sm.deadline_ns = p.wait_ns;
+    sm.status = p.status;
+    for (int i = 0; i < 20; ++i) sm.rk[i] = p.round_key[i];
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
@@ -1425,362 +1534,317 @@ __global__ void __launch_bounds__(kThreads, 2) rows_kernel(const __grid_constant
   // stream was still finishing (launch latency, block start-up and the set-up above then overlap with that
   // kernel's tail).  Nothing in global memory may be touched before the wait below, which returns once the
   // earlier kernel has completed and its writes are visible; the grid behind this one may start likewise.
-  asm volatile("griddepcontrol.wait;" ::: "memory");
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-
-  const int full_end = (int)(p.V & ~(int64_t)15);  // entries covered by full groups
+  asm volatile("griddepcontrol.wait;" ::: "memory");
 
   if (warp < kStreamWarps) {
     // ------------------------------------------------------------------ consumers
-    SegIter it(p, true);
-    Seg s;
-    RowInfo ri;
-    uint32_t stage = 0, phase = 0;  // ring position
-    uint32_t n = 0;                 // segments handed to the finishing warp so far
-    const uint32_t *const rk = p.round_key;
-    unsigned char *const queue = dyn + (RING ? kStages * kStageBytes : 0) + warp * F::kQueueBytes;
-    // sampler 1: the warp's lane sums of the last kLB steps
-    float *const bscratch = reinterpret_cast<float *>(dyn + (RING ? kStages * kStageBytes : 0)) + warp * (F::kLB * 32);
-    // vector order of this lane inside its 64 bytes (the lanes of a quarter warp hit distinct banks)
-    const int rot = (lane >> 1) & 3;
-    while (it.next(p, s, ri)) {
-      if (ri.masked) continue;
-      if (ri.invalid) {
-        // nothing to compute, but the row's chunks are on their way: let them pass
-        if (RING) {
-          const int nc = s.e_hi > s.e_lo ? (s.e_hi - s.e_lo + kChunkE - 1) / kChunkE : 0;
-          for (int c = 0; c < nc; ++c) {
-            mbar_wait(&sm.full[stage], phase, sm);
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&sm.empty[stage]);
-            if (++stage == kStages) { stage = 0; phase ^= 1u; }
-          }
-        }
-        continue;
-      }
-      const char *row = row_ptr<DT>(p, s.row);
-      const uint32_t grow = p.row_base + (uint32_t)s.row;
+    const uint32_t ring_warp = ring + (uint32_t)warp * (kNS * kWarpBytes);
+    uint32_t slot = 0, phase = 0;   // ring position
+    uint32_t n = 0;                 // row pieces handed to the finishing warp so far
+    const uint32_t *const rk = sm.rk;
+    unsigned char *const queue = dyn + kStreamWarps * kNS * kWarpBytes + warp * QueueBytes<DT>::value;
+    const uint32_t rec_warp = ring + kStreamWarps * kNS * kWarpBytes + (uint32_t)warp * kRecordBytesPerWarp;  // sampler 1
+    const int r8 = lane & 7;        // vector order of this lane inside its 128 bytes
+    const int ga = r8 / F::kVG;     // ... and the resulting order of its groups
+    Acc acc;
+    acc_reset(acc);
+    Best best;
+    float gy = -CUDART_INF_F;  // greedy rows without sampler 0: the lane's largest logit and its index
+    int gi = -1;
+    float ethr = 0.f, c = 0.f, tau = 0.f;
+    float zmax = -CUDART_INF_F;  // GAP: the lane's largest logit of the row piece
+    int err = 0, qn = 0, it = 0;
+    bool greedy = false, unusable = false;
+    for (;;) {
+      // a wait that was given up ends the warp's work: the slot's record cannot be trusted then
+      if (__any_sync(0xffffffffu, !mbar_wait(&sm.full[warp][slot], phase, sm))) break;
+      const SliceMeta m = sm.meta[warp][slot];
+      if (m.flags & kFlagEnd) break;
       const uint32_t seg = n + 1;
-#define E3_MAKE_CTX(ex)                                                                                  \
-  EvalCtx ex;                                                                                            \
-  ex.rk = rk; ex.row = row; ex.tau = ri.tau; ex.slack_k = p.slack_scale; ex.grow = grow; ex.ctr_lo = p.ctr_lo; \
-  ex.ctr_hi8 = p.ctr_hi8;                                                                                \
+      const char *const row = row_ptr<DT>(p, m.row);
+      const uint32_t grow = p.row_base + (uint32_t)m.row;
+#define E3_MAKE_CTX(ex)                                                                                 \
+  EvalCtx ex;                                                                                           \
+  ex.rk = rk; ex.row = row; ex.tau = tau; ex.slack_k = p.slack_scale; ex.grow = grow; ex.ctr_lo = p.ctr_lo; \
+  ex.ctr_hi8 = p.ctr_hi8;                                                                               \
   ex.seg = seg; ex.V = (int)p.V
 
-      Acc acc;
-      acc_reset(acc);
-      Best best;
-      best.y[0] = best.y[1] = best.y[2] = -CUDART_INF_F;
-      best.b[0] = best.b[1] = best.b[2] = -1;
-      best.zf = 0.f;
-      set_gate(best, enc_neg_inf(), ri.tau);
-      float ethr = 0.f;
-      int err = 0, qn = 0;
-      BlockState bs;
-      block_state_reset(bs);
-
-      const int nchunks = s.e_hi > s.e_lo ? (s.e_hi - s.e_lo + kChunkE - 1) / kChunkE : 0;
-      const int fast_end = s.e_hi < full_end ? s.e_hi : full_end;  // full groups of the piece end here
-      const bool stream = RING && !ri.greedy;
-#pragma unroll 1
-      for (int c = 0; c < nchunks; ++c) {
-        const int cs = s.e_lo + c * kChunkE;
-        const int e_lane = cs + tid * kLaneE;
-        const unsigned char *stage_ptr = nullptr;
-        if (RING) {
-          mbar_wait(&sm.full[stage], phase, sm);
-          stage_ptr = ring + (size_t)stage * kStageBytes;
+      if (m.flags & kFlagFirst) {
+        tau = m.tau;
+        greedy = p.mode == kModeSample && tau == 0.f;
+        unusable = !greedy && !(tau > 0.f && tau < CUDART_INF_F);
+        c = greedy || unusable ? 0.f : __fdiv_rn(kLog2e, tau);
+        acc_reset(acc);
+        gy = -CUDART_INF_F; gi = -1;
+        zmax = -CUDART_INF_F;
+        if (SAMPLER == 0) {
+          best.y[0] = best.y[1] = best.y[2] = -CUDART_INF_F;
+          best.b[0] = best.b[1] = best.b[2] = -1;
+          best.zf = 0.f;
+          set_gate(best, enc_neg_inf(), tau);
+          ethr = 0.f;
         }
-        if (stream) {
-          const unsigned char *lane_data = stage_ptr + tid * kLaneBytes;
-          const int lim = fast_end < cs + kChunkE ? fast_end : cs + kChunkE;
-          if (c == 0) {
-            float R0;
+        err = unusable ? kErrValue : 0;
+        qn = 0; it = 0;
+      }
+      if (m.n > 0 && !unusable) {
+        const uint32_t lane_addr = ring_warp + slot * kWarpBytes + (uint32_t)(lane * kLaneBytes);
+        if (!p.bulk || (((uint32_t)m.n * kEsize) & 15u) != 0u)
+          patch_slice<DT>(row, m.s_lo, m.n, p.bulk != 0, ring_warp + slot * kWarpBytes, lane);
+        const int e_lane = m.s_lo + lane * kLaneE;
+        const int nlane = m.n - lane * kLaneE < 0 ? 0 : (m.n - lane * kLaneE > kLaneE ? kLaneE : m.n - lane * kLaneE);
+        const uint32_t B = lane_addr | (uint32_t)(r8 << 4);
+        if (greedy) {
+          GreedyIO g;
+          g.y = SAMPLER == 0 ? best.y[0] : gy;
+          g.i = SAMPLER == 0 ? best.b[0] : gi;
+          g.err = err;
+          turn_greedy<DT>(g, B, e_lane, nlane, r8);
+          if (SAMPLER == 0) { best.y[0] = g.y; best.b[0] = g.i; } else { gy = g.y; gi = g.i; }
+          err = g.err;
+        } else {
+          f2 Zt2, Wt2;
+          float Zg[kG];
+          float zturn = -CUDART_INF_F;
+          bool done = false;
+          const bool full = m.n >= F::kWarpE;
+          if (full && acc.R > -CUDART_INF_F) {
+            if (SAMPLER == 0 && (it & 3) == 0) {
+              const int enc = read_best(sm, seg);
+              if (enc > best.enc) {
+                set_gate(best, enc, tau);
+                ethr = gate_threshold(best.enc, acc.nRc);
+              }
+            }
             if (SAMPLER == 0) {
-              SeedIO sd;
-              sd.best = best;
-              E3_MAKE_CTX(ex);
-              seed_piece<DT, SAMPLER>(sd, ex, lane_data, e_lane, lim, sm);
-              best = sd.best;
-              R0 = sd.R0;
+              uint4 v[8];
+              load_slice(B, v);
+              slice_sums<DT, true, false>(v, pack2f(c, c), pack2f(acc.nRc, acc.nRc), Zt2, Wt2, Zg);
+              if (GAP) zturn = slice_max<DT>(v);
             } else {
-              R0 = seed_reference<DT>(lane_data, e_lane, lim);
+              slice_sums_rolled<DT, GAP>(B, pack2f(c, c), pack2f(acc.nRc, acc.nRc), Zt2, Wt2, zturn);
             }
-            if (R0 > -CUDART_INF_F) {
-              const float nRc = -R0 * ri.c;
-              if (fabsf(nRc) < CUDART_INF_F) { acc.R = R0; acc.nRc = nRc; }
+            const float Zs = sum2(Zt2), Ws = sum2(Wt2);
+            const bool bad = !(Zs <= kTurnSumMax) || !(fabsf(Ws) <= kTurnWMax);
+            done = !__any_sync(0xffffffffu, bad);
+          }
+          if (!done) {
+            const bool fresh = acc.R == -CUDART_INF_F;
+            {
+              CarefulIO<DT> io;
+              io.acc = acc; io.err = err;
+              turn_careful<DT, SAMPLER == 0>(io, B, nlane, r8, c);
+              acc = io.acc; err = io.err; Zt2 = io.Zt2; Wt2 = io.Wt2; zturn = io.zmax;
+              if (SAMPLER == 0) {
+#pragma unroll
+                for (int j = 0; j < kG; ++j) Zg[j] = io.Zg[j];
+              }
             }
-            if (SAMPLER == 0) ethr = gate_threshold(best.enc, acc.nRc);
-          } else if (SAMPLER == 0 && (c & 3) == 0) {
-            const int enc = read_best(sm, seg);
-            if (enc > best.enc) {
-              set_gate(best, enc, ri.tau);
+            if (SAMPLER == 0) {
+              if (fresh && full && acc.R > -CUDART_INF_F) {
+                E3_MAKE_CTX(ex);
+                Best tb = best;
+                seed_gate<DT>(tb, ex, lane_addr, e_lane, sm);
+                best = tb;
+              }
               ethr = gate_threshold(best.enc, acc.nRc);
             }
           }
-          // the row's last, partial group (V not a multiple of 16) sits behind the full groups of this chunk
-          float zextra = 0.f;
-          const bool tail_here = fast_end < s.e_hi && fast_end >= cs && fast_end < cs + kChunkE;
-          if (tail_here) {
-            const int owner = (fast_end - cs) / kLaneE;  // thread whose 64 bytes would hold it
-            if ((owner >> 5) == warp) {
-              SlowIO io;
-              io.acc = acc; io.err = err; io.zsum = 0.f;
-              if (SAMPLER == 0) io.best = best;
-              E3_MAKE_CTX(ex);
-              slow_groups<DT, SAMPLER, true>(io, ex, owner == tid ? fast_end : s.e_hi, s.e_hi, ri.c, sm);
-              acc = io.acc; err = io.err;
-              if (SAMPLER == 0) best = io.best;
-              zextra = io.zsum;
-              if (SAMPLER == 0) ethr = gate_threshold(best.enc, acc.nRc);
-            }
-          }
-          // ---- the streaming form: one group of 16 entries per turn (a single copy of the code, so that
-          // the loop stays in the instruction cache).  Turn gi works on group gi ^ ga of the thread's 64
-          // bytes and reads its vectors in the order i ^ rot, which keeps the lanes of a quarter warp on
-          // distinct banks.  All lanes of the warp share one reference logit.
-          const int ga = kG == 2 ? (rot >> 1) : 0;
-          float zl = zextra;  // sampler 1: this thread's share of its block
-          // Without the per-group work of sampler 0, a stage that lies wholly inside the row is taken in
-          // one piece: the thread's 64 bytes in straight-line code and one check for the warp.  If the
-          // check fails (stale reference, a value that is not finite) nothing has been added yet and
-          // the turns below deal with the stage.
-          bool stage_done = false;
-          if (SAMPLER != 0 && fast_end >= cs + kChunkE) {
-            uint4 raw[4];
-            const uint4 *pv = reinterpret_cast<const uint4 *>(lane_data);
+          acc.Z2 = add2(acc.Z2, Zt2);
+          acc.W2 = add2(acc.W2, Wt2);
+          if (GAP) zmax = fmaxf(zmax, zturn);
+          if (SAMPLER == 0) {
 #pragma unroll
-            for (int i = 0; i < 4; ++i) raw[i] = pv[i ^ rot];
-            f2 Zs2, Ws2;
-            const float Zs = hot_vectors<DT, 4>(raw, pack2f(ri.c, ri.c), pack2f(acc.nRc, acc.nRc), Ws2, Zs2);
-            if (!__any_sync(0xffffffffu, !(Zs <= kGroupSumMax))) {
-              acc.Z2 = add2(acc.Z2, Zs2);
-              acc.W2 = add2(acc.W2, Ws2);
-              zl += Zs;
-              stage_done = true;
-            }
-          }
-#pragma unroll 1
-          for (int gi = stage_done ? kG : 0; gi < kG; ++gi) {
-            const int gn = gi ^ ga;
-            const int g0 = e_lane + (gn << 4);
-            const bool have = g0 + kGroup <= lim;
-            uint4 raw[kVG];
-            {
-              const uint4 *pv = reinterpret_cast<const uint4 *>(lane_data) + gn * kVG;
-#pragma unroll
-              for (int i = 0; i < kVG; ++i) raw[i] = pv[(i ^ rot) & (kVG - 1)];
-            }
-            float Zg = 0.f;
-            f2 Zg2 = pack2f(0.f, 0.f), Wg2 = pack2f(0.f, 0.f);  // the group's sums; they join the state once they are known to be sound
-#pragma unroll 1
-            for (int attempt = 0;; ++attempt) {
-              if (have) Zg = hot_group<DT>(raw, pack2f(ri.c, ri.c), pack2f(acc.nRc, acc.nRc), Wg2, Zg2);
-              if (!__any_sync(0xffffffffu, have && !(Zg <= kGroupSumMax))) break;
-              // the reference is stale for some lane (or a value is not finite)
-              const float gm = have ? group_max<DT>(raw) : -CUDART_INF_F;
-              const float newR = dec_float(__reduce_max_sync(0xffffffffu, enc_float(gm)));
-              const float nRc = -newR * ri.c;
-              if (attempt == 0 && newR > acc.R && newR < CUDART_INF_F && fabsf(nRc) < CUDART_INF_F) {
-                // move the warp's reference up to the largest logit of this turn and repeat the group
-                const float d = nRc - acc.nRc;
-                const float f = acc.R == -CUDART_INF_F ? 0.f : ex2f(d);
-                const f2 ff = pack2f(f, f);
-                acc.W2 = mul2(ff, fma2(pack2f(d, d), acc.Z2, acc.W2));
-                acc.Z2 = mul2(ff, acc.Z2);
-                if (f == 0.f) acc.Z2 = acc.W2 = pack2f(0.f, 0.f);
-                acc.R = newR; acc.nRc = nRc;
-                zl *= f;
-                if (SAMPLER == 0) ethr = gate_threshold(best.enc, acc.nRc);
-                continue;
-              }
-              // NaN, +inf or numbers outside the fp32 range: the careful form sorts it out
-              StepIO io;
-              io.acc = acc; io.err = err; io.Zextra = zl;
-              io.Zg[0] = 0.f; io.Zg[kG - 1] = 0.f;
-              redo_step<DT, true>(io, lane_data, have ? (1 << gn) : 0, ri.c);
-              acc = io.acc; err = io.err; zl = io.Zextra;
-              Zg = io.Zg[gn];
-              Zg2 = Wg2 = pack2f(0.f, 0.f);  // the careful form has added the group already
-              if (SAMPLER == 0) ethr = gate_threshold(best.enc, acc.nRc);
-              break;
-            }
-            acc.Z2 = add2(acc.Z2, Zg2);
-            acc.W2 = add2(acc.W2, Wg2);
-            zl += Zg;
-            if (SAMPLER == 0) {
+            for (int j = 0; j < kG; ++j) {
+              const int g0 = e_lane + ((j ^ ga) << 4);
               const uint4 cb = philox(rk, (uint32_t)g0 >> 4, grow, p.ctr_lo, p.ctr_hi8 | 0u);
-              const bool over = Zg > ethr;
-              const bool flag = have && (any_ff4(cb) != 0u || over);
+              const bool over = Zg[j] > ethr;
+              const bool flag = g0 < m.s_lo + m.n && (any_ff4(cb) != 0u || over);
               const uint32_t ballot = __ballot_sync(0xffffffffu, flag);
               if (ballot != 0u) {
                 if (flag) {
                   const int pos = qn + __popc(ballot & ((1u << lane) - 1u));
                   reinterpret_cast<int *>(queue)[pos] = g0 | (over ? 1 : 0);
-                  uint4 *ent = reinterpret_cast<uint4 *>(queue + kQueueHdrBytes + pos * F::kEntryBytes);
-                  ent[0] = cb;
+                  uint4 *ent = reinterpret_cast<uint4 *>(queue + kQueueCap * 4 + pos * F::kEntryBytes);
+                  const uint32_t ga_addr = lane_addr + (uint32_t)((j ^ ga) << 4) * kEsize;
+                  const int left = m.s_lo + m.n - g0;  // entries of the group that belong to the row piece
 #pragma unroll
-                  for (int i = 0; i < kVG; ++i) ent[1 + ((i ^ rot) & (kVG - 1))] = raw[i];
+                  for (int i = 0; i < F::kVG; ++i) {
+                    uint4 q = lds128(ga_addr + 16 * i);
+                    if (left < kGroup) {  // the row ends inside the group: what lies behind it counts as -inf
+                      uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+                      for (int k = 0; k < 4; ++k) {
+                        if (DT == 1) {
+                          const int e = 8 * i + 2 * k;
+                          w[k] = (e < left ? (w[k] & 0xFFFFu) : 0xFF80u) | (e + 1 < left ? (w[k] & 0xFFFF0000u) : 0xFF800000u);
+                        } else {
+                          w[k] = 4 * i + k < left ? w[k] : 0xFF800000u;
+                        }
+                      }
+                      q = make_uint4(w[0], w[1], w[2], w[3]);
+                    }
+                    ent[i] = q;
+                  }
                 }
                 qn += __popc(ballot);
                 if (qn >= kDrainAt) {
                   Best tb = best;
-                  drain_queue<DT>(rk, grow, p.ctr_lo, p.ctr_hi8, ri.tau, p.slack_scale, seg, queue, qn, tb, sm);
+                  drain_queue<DT>(rk, grow, p.ctr_lo, p.ctr_hi8, tau, p.slack_scale, seg, queue, qn, tb, sm);
                   best = tb;
                   qn = 0;
                   const int enc = read_best(sm, seg);
-                  if (enc > best.enc) set_gate(best, enc, ri.tau);
+                  if (enc > best.enc) set_gate(best, enc, tau);
                   ethr = gate_threshold(best.enc, acc.nRc);
                 }
               }
             }
           }
-          if (SAMPLER == 1) block_step<DT>(zl, e_lane >> 8, acc.nRc, rk, grow, p.ctr_lo, p.ctr_hi8, bs, bscratch, lane, c);
-        } else if (ri.greedy) {
-          SlowIO io;
-          io.acc = acc; io.err = err; io.zsum = 0.f;
-          if (SAMPLER != 0) {  // the running maximum lives in the list of blocks, which greedy rows do not use
-            io.best.y[0] = bs.top.y[0]; io.best.b[0] = bs.top.b[0];
-          } else {
-            io.best = best;
+          if (SAMPLER == 1) {
+            // The lane's sum and the reference it refers to: into the record of this use of the slot.  The feeding
+            // lane ships the record to the workspace when it sees the slot freed (a global store from here would
+            // cost the warp microseconds while the copies keep the memory system busy).
+            const uint32_t rec = rec_warp + (phase * kNS + slot) * (uint32_t)(kRecordFloats * 4);
+            asm volatile("st.shared.f32 [%0], %1;" ::"r"(rec + (uint32_t)lane * 4u), "f"(sum2(Zt2)) : "memory");
+            if (lane == 0) asm volatile("st.shared.f32 [%0], %1;" ::"r"(rec + 128u), "f"(acc.nRc) : "memory");
+            fence_async_smem();
           }
-          greedy_groups<DT>(io, row, RING ? stage_ptr + tid * kLaneBytes : nullptr, e_lane,
-                            fast_end < cs + kChunkE ? fast_end : cs + kChunkE, s.e_hi);
-          err = io.err;
-          if (SAMPLER != 0) {
-            bs.top.y[0] = io.best.y[0]; bs.top.b[0] = io.best.b[0];
-          } else {
-            best = io.best;
-          }
-        } else {
-          // rows that cannot use the ring: everything through the guarded form
-          SlowIO io;
-          io.acc = acc; io.err = err; io.zsum = 0.f;
-          if (SAMPLER == 0) io.best = best;
-          E3_MAKE_CTX(ex);
-          slow_groups<DT, SAMPLER, true>(io, ex, e_lane < s.e_hi ? e_lane : s.e_hi, s.e_hi, ri.c, sm);
-          acc = io.acc; err = io.err;
-          if (SAMPLER == 0) best = io.best;
-          if (SAMPLER == 1) block_step<DT>(io.zsum, e_lane >> 8, acc.nRc, rk, grow, p.ctr_lo, p.ctr_hi8, bs, bscratch, lane, c);
         }
-        if (RING) {
-          __syncwarp();
-          if (lane == 0) mbar_arrive(&sm.empty[stage]);
-          if (++stage == kStages) { stage = 0; phase ^= 1u; }
-        }
+        ++it;
       }
-      if (SAMPLER == 0 && qn > 0) {
-        Best tb = best;
-        drain_queue<DT>(rk, grow, p.ctr_lo, p.ctr_hi8, ri.tau, p.slack_scale, seg, queue, qn, tb, sm);
-        best = tb;
-        qn = 0;
-      }
-      if (SAMPLER == 1 && !ri.greedy) {
-        // blocks of the unfinished round: lanes whose step has not come hold no block (b = -1)
-        block_flush<DT>(rk, grow, p.ctr_lo, p.ctr_hi8, bs, bscratch, lane);
-      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&sm.empty[warp][slot]);  // the slot is free again
+      if (++slot == kNS) { slot = 0; phase ^= 1u; }
 
-      AccS fin = to_scalar(acc);
-      if (!ri.greedy) {
-        // NaN or infinite sums (a NaN or +inf logit, or numbers outside the fp32 range): settle this
-        // thread's entries of the piece with the careful form, which also says what was wrong
-        const bool odd = !(fabsf(fin.Z) < CUDART_INF_F) || !(fabsf(fin.W) < CUDART_INF_F);
-        if (__any_sync(0xffffffffu, odd)) {
-          fin.R = -CUDART_INF_F; fin.nRc = kNoRef; fin.Z = fin.W = 0.f;
-#pragma unroll 1
-          for (int g = 0; g < nchunks * kG; ++g) {
-            const int e0 = s.e_lo + (g / kG) * kChunkE + tid * kLaneE + (g % kG) * kGroup;
-            if (e0 < s.e_hi) {
-              float z[16];
-              load_group_guarded<DT>(row, e0, e0 + kGroup <= (int)p.V ? 16 : (int)p.V - e0, z);
-              careful_accumulate(fin, z, ri.c, -CUDART_INF_F, err);
-            }
-          }
+      if (m.flags & kFlagLast) {
+        if (SAMPLER == 0 && qn > 0) {
+          Best tb = best;
+          drain_queue<DT>(rk, grow, p.ctr_lo, p.ctr_hi8, tau, p.slack_scale, seg, queue, qn, tb, sm);
+          best = tb;
+          qn = 0;
         }
-      }
-
-      // warp-level merge, hand-over to the finishing warp
-      Piece pw;
-      pw.M = -fin.nRc; pw.Z = fin.Z; pw.W = fin.W;
-      if (fin.R == -CUDART_INF_F) { pw.M = 0.f; pw.Z = 0.f; pw.W = 0.f; }
-      pw.zf = SAMPLER == 0 ? best.zf : 0.f; pw.err = err;
-      if (SAMPLER == 0) {  // the thread's leaders; sampler 1 has its blocks there (greedy rows: the maximum) already
+        // warp-level merge (all lanes share the reference), hand-over to the finishing warp
+        float Zs = sum2(acc.Z2), Ws = sum2(acc.W2);
+        if (!(fabsf(Zs) < CUDART_INF_F) || !(fabsf(Ws) < CUDART_INF_F)) err |= kErrValue;
 #pragma unroll
-        for (int i = 0; i < 3; ++i) { bs.top.y[i] = best.y[i]; bs.top.b[i] = best.b[i]; }
-      }
-      warp_merge(pw, bs.top, SAMPLER >= 0);
-      const uint32_t slot = n % kSlots, use = n / kSlots;
-      if (use > 0) mbar_wait(&sm.wfree[slot], (use - 1) & 1u, sm);
-      if (lane == 0) {
-        WarpPartial &w = sm.wpart[slot][warp];
-        w.M = pw.M; w.Z = pw.Z; w.W = pw.W; w.err = pw.err; w.zf = pw.zf;
+        for (int o = 16; o > 0; o >>= 1) {
+          Zs += __shfl_xor_sync(0xffffffffu, Zs, o);
+          Ws += __shfl_xor_sync(0xffffffffu, Ws, o);
+        }
+        err = __reduce_or_sync(0xffffffffu, err);
+        float zf = 0.f;
+        Top3 wtop;
+        top3_reset(wtop);
+        if (SAMPLER == 0) {  // the thread's leaders
 #pragma unroll
-        for (int i = 0; i < 3; ++i) { w.ty[i] = bs.top.y[i]; w.tb[i] = bs.top.b[i]; }
-        mbar_arrive(&sm.wfull[slot]);
+          for (int i = 0; i < 3; ++i) { wtop.y[i] = best.y[i]; wtop.b[i] = best.b[i]; }
+          zf = best.zf;
+        } else if (SAMPLER == 1 && greedy) {  // the lane's maximum
+          wtop.y[0] = gy; wtop.b[0] = gi;
+        }
+        if (SAMPLER == 0 || (SAMPLER == 1 && greedy)) warp_merge_top(wtop, zf);
+        const float zm = GAP ? dec_float(__reduce_max_sync(0xffffffffu, enc_float(zmax))) : 0.f;
+        const uint32_t hslot = n % kSlots, use = n / kSlots;
+        if (use > 0 && __any_sync(0xffffffffu, !mbar_wait(&sm.wfree[hslot], (use - 1) & 1u, sm))) break;
+        if (lane == 0) {
+          WarpPartial &w = sm.wpart[hslot][warp];
+          const bool has = acc.R > -CUDART_INF_F;
+          w.M = has ? -acc.nRc : 0.f; w.Z = has ? Zs : 0.f; w.W = has ? Ws : 0.f; w.err = err; w.zf = zf;
+          w.zmax = zm;
+#pragma unroll
+          for (int i = 0; i < 3; ++i) { w.ty[i] = wtop.y[i]; w.tb[i] = wtop.b[i]; }
+          mbar_arrive(&sm.wfull[hslot]);
+        }
+        ++n;
       }
-      ++n;
     }
 #undef E3_MAKE_CTX
   } else if (warp == kStreamWarps) {
-    // ------------------------------------------------------------------ producer (one thread)
-    if (RING && lane == 0) {
-      SegIter it(p, false);
-      Seg s;
-      RowInfo ri;
-      uint32_t cc = 0, stage = 0, phase = 1;  // phase: parity of the previous use of the stage
-      while (it.next(p, s, ri)) {
-        if (ri.masked) continue;
-        const char *row = row_ptr<DT>(p, s.row);
-        const int nchunks = s.e_hi > s.e_lo ? (s.e_hi - s.e_lo + kChunkE - 1) / kChunkE : 0;
-        const int lim = s.e_hi < full_end ? s.e_hi : full_end;
-        for (int c = 0; c < nchunks; ++c) {
-          if (cc >= (uint32_t)kStages) mbar_wait(&sm.empty[stage], phase, sm, 32u);
-          const int cs = s.e_lo + c * kChunkE;
-          const int ce = cs + kChunkE < lim ? cs + kChunkE : lim;
-          const uint32_t bytes = ce > cs ? (uint32_t)(ce - cs) * kEsize : 0u;
-          const bool dead = *reinterpret_cast<volatile int *>(&sm.timeout) != 0;
-          if (bytes > 0 && !dead) {
-            mbar_arrive_expect_tx(&sm.full[stage], bytes);
-            bulk_copy_g2s(ring + (size_t)stage * kStageBytes, row + (size_t)cs * kEsize, bytes, &sm.full[stage]);
-          } else {
-            mbar_arrive(&sm.full[stage]);
+    // ------------------------------------------------------------------ feeding warp: lane w feeds consumer warp w
+    if (lane < kStreamWarps) {
+      constexpr unsigned kLanes = (1u << kStreamWarps) - 1u;
+      const uint32_t ring_w = ring + (uint32_t)lane * (kNS * kWarpBytes);
+      Feeder<DT> feeder(p);
+      uint32_t issued = 0, slot = 0, phase = 1;  // phase: parity of the previous use of the slot
+      // Sampler 1: ships the record the consumer warp left for the use `par` of slot `st` (the slot's record still
+      // describes that use).  A record's buffer comes round again six uses later; by then its bulk store has read it
+      // (all but the two most recent stores of this thread have, before a new one is issued).
+      const uint32_t rec_lane = ring + kStreamWarps * kNS * kWarpBytes + (uint32_t)lane * kRecordBytesPerWarp;
+      auto ship = [&](uint32_t st, uint32_t par) {
+        const SliceMeta &pm = sm.meta[lane][st];
+        if (pm.n > 0 && !(pm.flags & kFlagEnd)) {
+          bulk_wait_read<2>();
+          const int64_t ti = pm.row * p.tiles_per_row + pm.s_lo / F::kWarpE;
+          bulk_store_s2g(p.ws_records + ti * kRecordFloats, rec_lane + (par * kNS + st) * (uint32_t)(kRecordFloats * 4),
+                         kRecordFloats * 4);
+        }
+      };
+      unsigned long long idle_since = 0;         // 0: the last pass over the lanes fed something
+      uint32_t idle_passes = 0;
+      while (__any_sync(kLanes, !feeder.done)) {
+        if (timed_out(sm)) break;  // somebody gave up: nothing more is fed, the consumers run out on their next wait
+        bool ready = false;
+        if (!feeder.done) {
+          ready = issued < (uint32_t)kNS;
+          if (!ready) {
+            uint32_t ok;
+            asm volatile("{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                         : "=r"(ok) : "r"(smem_addr(&sm.empty[lane][slot])), "r"(phase) : "memory");
+            ready = ok != 0;
           }
-          ++cc;
-          if (++stage == kStages) { stage = 0; phase ^= 1u; }
+          if (ready) {
+            if (SAMPLER == 1 && issued >= (uint32_t)kNS) ship(slot, phase);
+            feeder.feed(p, sm, ring_w, lane, (int)slot);
+            if (!feeder.stalled) {
+              ++issued;
+              if (++slot == kNS) { slot = 0; phase ^= 1u; }
+            }
+          }
+        }
+        if (__any_sync(kLanes, ready)) {
+          idle_since = 0;
+          idle_passes = 0;
+        } else if ((++idle_passes & 255u) == 0u) {  // no consumer has freed a slot for a while: look at the clock
+          const unsigned long long now = global_ns();
+          if (idle_since == 0) idle_since = now;
+          if (now - idle_since > p.wait_ns) raise_timeout(sm);
         }
       }
-      // Before leaving, see every copy still in flight land (bounded).
-      const uint32_t back = cc < (uint32_t)kStages ? cc : (uint32_t)kStages;
-      for (uint32_t q = cc - back; q < cc; ++q) {
-        const uint32_t st = q % kStages, round = q / kStages;
-        for (uint32_t i = 0; i < kSpinLimit && !mbar_try_wait(&sm.full[st], round & 1u); ++i) __nanosleep(64);
+      // Before leaving, see every copy still in flight land (bounded): the slots handed out last.
+      {
+        const uint32_t back = issued < (uint32_t)kNS ? issued : (uint32_t)kNS;
+        const unsigned long long t0 = global_ns();
+        for (uint32_t q = issued - back; q < issued; ++q) {
+          const uint32_t st = q % kNS, round = q / kNS;
+          for (uint32_t i = 1; !mbar_try_wait(&sm.full[lane][st], round & 1u); ++i)
+            if ((i & 63u) == 0u && global_ns() - t0 > p.wait_ns) break;
+        }
+        if (SAMPLER == 1) {  // ... and the records of those slots, once the consumer warp is done with them
+          for (uint32_t q = issued - back; q < issued; ++q) {
+            const uint32_t st = q % kNS, round = q / kNS;
+            if (sm.meta[lane][st].flags & kFlagEnd) continue;
+            bool ok = true;
+            for (uint32_t i = 1; !mbar_try_wait(&sm.empty[lane][st], round & 1u); ++i)
+              if (timed_out(sm) || ((i & 63u) == 0u && global_ns() - t0 > p.wait_ns)) { ok = false; break; }
+            if (ok) ship(st, round & 1u);
+          }
+          bulk_wait_all();
+        }
       }
     }
   } else {
     // ------------------------------------------------------------------ finishing warp
-    SegIter it(p, true, true);
+    SegIter<DT> sit(p, true);
     Seg s;
     RowInfo ri;
     uint32_t n = 0;
     u64 *const pieces = reinterpret_cast<u64 *>(p.ws_pieces);
     constexpr int kPieceStride = (int)(kPieceBytes / 8);
     const bool sample = p.mode == kModeSample;
-    // The code below runs once or twice per CTA, the last time at the very end of the CTA's life, when
-    // nothing hides it, and a first run through cold code is dominated by instruction fetches (several
-    // times the warm time).  So the warp rehearses it while the consumers work on the first piece: pass
-    // number p.rehearse takes the first piece's descriptors and made-up sums through the same
-    // instructions with every store, barrier operation and workspace write switched off.  (The pass number
-    // is a kernel argument so that the compiler keeps a single copy of the loop body.)
-    for (int pass = 0;; ++pass) {
-      const bool ghost = pass == p.rehearse;
-      if (ghost) {
-        SegIter peek = it;
-        if (!peek.next(p, s, ri)) continue;
-      } else if (!it.next(p, s, ri)) {
-        break;
-      }
-      if (ri.masked || ri.invalid) {
-        if (!ghost && s.starts && lane == 0) write_skipped(p, s.row, ri);
+    while (sit.next(p, s, ri)) {
+      if (ri.masked) {
+        if (s.starts && lane == 0) write_skipped(p, s.row, ri);
         continue;
       }
       // the target's logit is fetched while the consumers work on the piece
@@ -1790,54 +1854,96 @@ __global__ void __launch_bounds__(kThreads, 2) rows_kernel(const __grid_constant
         target = __ldg(p.targets + s.row);
         if (target >= 0 && target < p.V) zt = load_elem<DT>(row_ptr<DT>(p, s.row), target);
       }
+      // A piece of a cut row: while the consumers still work on it, look for the row's other pieces.  When all
+      // of them are there already, this CTA is the last one to arrive and finishes the row as soon as its own
+      // piece is complete, without publishing it: the others have looked for it in vain and have given up.
+      const int span = s.whole ? 0 : s.k1 - s.k0 + 1;
+      const int kmine = s.k0 + lane;  // the CTA whose piece this lane looks after (rows held by up to 32 CTAs)
+      Piece early;
+      bool early_ok = false;
+      if (!s.whole && span <= 32) {
+        bool ok = true;
+        if (lane < span && kmine != (int)blockIdx.x) {
+          const bool is_first_seg = quot(p, first_tile_of(p, kmine), p.tiles_per_row) == s.row;
+          ok = piece_load(pieces + ((size_t)kmine * 2 + (is_first_seg ? 0 : 1)) * kPieceStride, p.call_id, early);
+        }
+        early_ok = __all_sync(0xffffffffu, ok);
+      }
       const uint32_t slot = n % kSlots, use = n / kSlots;
-      if (!ghost) mbar_wait_warp(&sm.wfull[slot], use & 1u, sm, lane);
+      if (!mbar_wait_warp(&sm.wfull[slot], use & 1u, sm, lane)) {
+        // A wait of this CTA ran out: it gives up on this piece and on all that follow.  Nobody else can finish
+        // these rows (a cut row needs this CTA's piece, which is never published), so they are marked here.
+        do {
+          if (lane == 0) {
+            if (!ri.masked) write_abandoned(p, s.row, SAMPLER == 1);
+            else if (s.starts) write_skipped(p, s.row, ri);
+          }
+        } while (sit.next(p, s, ri));
+        break;
+      }
+      if (!s.whole && span <= 32 && !early_ok) {  // a second look, now that the own piece is complete
+        bool ok = true;
+        if (lane < span && kmine != (int)blockIdx.x) {
+          const bool is_first_seg = quot(p, first_tile_of(p, kmine), p.tiles_per_row) == s.row;
+          ok = piece_load(pieces + ((size_t)kmine * 2 + (is_first_seg ? 0 : 1)) * kPieceStride, p.call_id, early);
+        }
+        early_ok = __all_sync(0xffffffffu, ok);
+      }
       Piece pc;
-      pc.M = 0.f; pc.Z = 0.f; pc.W = 0.f; pc.zf = 0.f; pc.err = 0; pc.pad = 0;
+      pc.M = 0.f; pc.Z = 0.f; pc.W = 0.f; pc.zf = 0.f; pc.err = 0; pc.zmax = -CUDART_INF_F;
       Top3 top;
       top3_reset(top);
-      if (!ghost && lane < kStreamWarps) {
+      if (lane < kStreamWarps) {
         const WarpPartial &w = sm.wpart[slot][lane];
-        pc.M = w.M; pc.Z = w.Z; pc.W = w.W; pc.err = w.err; pc.zf = w.zf;
+        pc.M = w.M; pc.Z = w.Z; pc.W = w.W; pc.err = w.err; pc.zf = w.zf; pc.zmax = w.zmax;
         if (SAMPLER >= 0) {
 #pragma unroll
           for (int i = 0; i < 3; ++i) { top.y[i] = w.ty[i]; top.b[i] = w.tb[i]; }
         }
       }
       __syncwarp();
-      if (!ghost) {
-        if (lane == 0) mbar_arrive(&sm.wfree[slot]);
-        ++n;
-      }
+      if (lane == 0) mbar_arrive(&sm.wfree[slot]);
+      ++n;
       // The order of every merge below is fixed by lane and piece numbers alone, so the result does not
-      // depend on which CTA ends up finishing the row.
-      warp_merge(pc, top, SAMPLER >= 0);
-      if (*reinterpret_cast<volatile int *>(&sm.timeout)) pc.err |= kErrTimeout;
+      // depend on which CTA ends up finishing the row, nor on the way it got hold of the pieces.
+      warp_merge(pc, top, false);
+      if (SAMPLER == 0 || (SAMPLER == 1 && ri.greedy)) warp_merge_top(top, pc.zf);
+      if (timed_out(sm)) pc.err |= kErrTimeout;
       bool fin = s.whole;
-      if (!s.whole || (ghost && pieces != nullptr)) {
-        // A piece of a cut row.  Store it, then (after a sequentially consistent fence) look for the
-        // row's other pieces: of all CTAs that hold a piece, the one whose fence comes last is sure to
-        // find them all and finishes the row.  Two CTAs may both find all pieces; they then write the
-        // same values.  Nobody waits for anybody.
-        if (lane == 0 && !ghost) {
+      if (!s.whole) {
 #pragma unroll
-          for (int i = 0; i < 3; ++i) { pc.ty[i] = top.y[i]; pc.tb[i] = top.b[i]; }
-          piece_store(pieces + ((size_t)blockIdx.x * 2 + (s.first ? 0 : 1)) * kPieceStride, p.call_id, pc);
-          asm volatile("fence.sc.gpu;" ::: "memory");
+        for (int i = 0; i < 3; ++i) { pc.ty[i] = top.y[i]; pc.tb[i] = top.b[i]; }
+        const Piece own = pc;
+        if (!early_ok) {
+          // Store the piece, then (after a sequentially consistent fence) look for the row's other pieces: of
+          // all CTAs that hold a piece, the one whose fence comes last is sure to find them all and finishes
+          // the row.  Two CTAs may both find all pieces; they then write the same values.  Nobody waits for
+          // anybody.
+          if (lane == 0) {
+            piece_store(pieces + ((size_t)blockIdx.x * 2 + (s.slot0 ? 0 : 1)) * kPieceStride, p.call_id, own);
+            asm volatile("fence.sc.gpu;" ::: "memory");
+          }
+          __syncwarp();
         }
-        __syncwarp();
-        pc.M = 0.f; pc.Z = 0.f; pc.W = 0.f; pc.zf = 0.f; pc.err = 0;
+        pc.M = 0.f; pc.Z = 0.f; pc.W = 0.f; pc.zf = 0.f; pc.err = 0; pc.zmax = -CUDART_INF_F;
         top3_reset(top);
         bool ok = true;
         for (int k = s.k0 + lane; k <= s.k1; k += 32) {
-          // CTA k keeps this row's piece in slot 0 when the row is the first thing it works on
-          const bool is_first_seg = quot(p, first_tile_of(p, k), p.tiles_per_row) == s.row;
           Piece q;
-          if (!piece_load(pieces + ((size_t)k * 2 + (is_first_seg ? 0 : 1)) * kPieceStride, p.call_id, q)) {
-            ok = false;
-            break;
+          if (k == (int)blockIdx.x) {
+            q = own;
+          } else if (early_ok) {
+            q = early;
+          } else {
+            // CTA k keeps this row's piece in slot 0 when the row is the first thing in its run
+            const bool is_first_seg = quot(p, first_tile_of(p, k), p.tiles_per_row) == s.row;
+            if (!piece_load(pieces + ((size_t)k * 2 + (is_first_seg ? 0 : 1)) * kPieceStride, p.call_id, q)) {
+              ok = false;
+              break;
+            }
           }
           pc.err |= q.err;
+          pc.zmax = fmaxf(pc.zmax, q.zmax);
           merge_stats_f(pc.M, pc.Z, pc.W, q.M, q.Z, q.W);
           if (SAMPLER >= 0) {
             if (q.tb[0] >= 0 && best_before(q.ty[0], q.tb[0], top.y[0], top.b[0])) pc.zf = q.zf;
@@ -1846,13 +1952,7 @@ __global__ void __launch_bounds__(kThreads, 2) rows_kernel(const __grid_constant
           }
         }
         fin = __all_sync(0xffffffffu, ok);
-        if (fin || ghost) warp_merge(pc, top, SAMPLER >= 0);
-      }
-      if (ghost) {  // made-up sums and a leader that exists in every row: entry 0 / block 0
-        fin = true;
-        pc.M = 0.f; pc.Z = 1.f; pc.W = 0.f; pc.zf = 0.f; pc.err = 0;
-        top3_reset(top);
-        top.y[0] = 0.f; top.b[0] = 0;
+        if (fin) warp_merge(pc, top, SAMPLER >= 0);
       }
       if (!fin) continue;
       int id = -1;
@@ -1861,23 +1961,113 @@ __global__ void __launch_bounds__(kThreads, 2) rows_kernel(const __grid_constant
         id = top.b[0];
         if (!ri.greedy && id >= 0) {
           EvalCtx ex;
-          ex.rk = p.round_key; ex.row = row_ptr<DT>(p, s.row); ex.tau = ri.tau; ex.slack_k = p.slack_scale;
+          ex.rk = sm.rk; ex.row = row_ptr<DT>(p, s.row); ex.tau = ri.tau; ex.slack_k = p.slack_scale;
           ex.grow = p.row_base + (uint32_t)s.row;
           ex.ctr_lo = p.ctr_lo; ex.ctr_hi8 = p.ctr_hi8; ex.seg = 0; ex.V = (int)p.V;
           if (SAMPLER == 1) {
-            // the whole warp settles the block and draws inside it
-            id = sample_in_blocks<DT>(ex, top, lane, zt);
+            // the token comes from block_sample_kernel
           } else {
             // fp32 scores decide unless the runner-up is within two slacks of the leader
             zt = pc.zf;
             const float slack2 = 2.f * fmaxf(score_slack(top.y[0], p.slack_scale), score_slack(top.y[1], p.slack_scale));
-            if (top.b[1] >= 0 && !(top.y[0] - top.y[1] > slack2)) id = settle_exact<DT>(ex, top, slack2, lane, zt);
+            if (top.b[1] >= 0 && !(top.y[0] - top.y[1] > slack2)) {
+              Top3 tcall = top;
+              float zcall = zt;
+              id = settle_exact<DT>(ex, tcall, slack2, lane, zcall);
+              zt = zcall;
+            }
           }
           have_zt = id >= 0;
         }
       }
-      if (lane == 0) finish_row(p, s.row, ri, pc.M, pc.Z, pc.W, id, pc.err, have_zt, zt, !ghost);
+      if (lane == 0) finish_row(p, s.row, ri, pc.M, pc.Z, pc.W, pc.zmax, id, pc.err, have_zt, zt, SAMPLER == 1);
+      if (!s.whole) {
+        // the row is done: nobody needs its pieces any more (a later run of this very launch must not find them)
+        for (int k = s.k0 + lane; k <= s.k1; k += 32) {
+          const bool is_first_seg = quot(p, first_tile_of(p, k), p.tiles_per_row) == s.row;
+          piece_wipe(pieces + ((size_t)k * 2 + (is_first_seg ? 0 : 1)) * kPieceStride, p.call_id);
+        }
+      }
     }
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Sampler 1, second kernel: one CTA of four warps per row.  It adds up the lanes of every block (the sums the
+// streaming kernel left in the workspace), turns the blocks into fp32 scores Y_b = L_b + g_b (one Philox call per
+// thread and round for four neighbouring blocks), keeps three leaders per thread, merges them, settles near-ties in
+// fp64 and draws the token inside the winning block by inverse CDF.  Rows the streaming kernel has finished itself
+// (greedy, flagged) are passed over.  It is launched behind the streaming kernel with programmatic stream
+// serialization, so its start-up overlaps that kernel's tail.
+// ---------------------------------------------------------------------------------------------
+constexpr int kSampleWarps = 4;
+template <int DT>
+__global__ void __launch_bounds__(kSampleWarps * 32) block_sample_kernel(const __grid_constant__ RowsParams p) {
+  using F = Fmt<DT>;
+  constexpr int kBS = F::kWarpE / 256;  // blocks per tile
+  constexpr int kLB = F::kLB;           // lanes per block
+  __shared__ uint32_t rk[20];
+  __shared__ float cand_y[kSampleWarps * 3];
+  __shared__ int cand_b[kSampleWarps * 3];
+  if (threadIdx.x < 20) rk[threadIdx.x] = p.round_key[threadIdx.x];
+  __syncthreads();
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int64_t row = blockIdx.x;
+  const float4 st = p.ws_rowstat[row];
+  if (st.z != 0.f) return;  // the whole block leaves: the record is the same for all its threads
+  const float tau = __ldg(p.temps + row);
+  const uint32_t grow = p.row_base + (uint32_t)row;
+  const int nblocks = (int)((p.V + 255) / 256);
+  const int ncalls = (nblocks + 3) / 4;
+  const float *const recs = p.ws_records + row * p.tiles_per_row * kRecordFloats;
+  Top3 top;
+  top3_reset(top);
+#pragma unroll 1
+  for (int q = threadIdx.x; q < ncalls; q += kSampleWarps * 32) {
+    const int b0 = 4 * q, tile = b0 / kBS, j0 = b0 % kBS;
+    const float ref = __ldg(recs + tile * kRecordFloats + 32);
+    const float4 *pp = reinterpret_cast<const float4 *>(recs + tile * kRecordFloats + j0 * kLB);
+    float4 v[kLB];
+#pragma unroll
+    for (int i = 0; i < kLB; ++i) v[i] = __ldg(pp + i);
+    const uint4 w = philox(rk, (uint32_t)q, grow, p.ctr_lo, p.ctr_hi8 | 2u);
+    const uint32_t xw[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      float S = 0.f;
+#pragma unroll
+      for (int i = 0; i < kLB / 4; ++i) {
+        const float4 u = v[k * (kLB / 4) + i];
+        S += (u.x + u.y) + (u.z + u.w);
+      }
+      // ln sum_i exp(s_i) + g_b, from S = sum 2^(z c + ref); a block without mass (or beyond the row) takes no part
+      if (b0 + k < nblocks && S > 0.f) top3_insert(top, (lg2f(S) - ref) * kLn2f + gumbel_from_word(xw[k]), b0 + k);
+    }
+  }
+  float zf = 0.f;
+  warp_merge_top(top, zf);
+  if (lane < 3) { cand_y[warp * 3 + lane] = lane == 0 ? top.y[0] : (lane == 1 ? top.y[1] : top.y[2]);
+                  cand_b[warp * 3 + lane] = lane == 0 ? top.b[0] : (lane == 1 ? top.b[1] : top.b[2]); }
+  __syncthreads();
+  if (warp != 0) return;
+  top3_reset(top);
+  if (lane < kSampleWarps * 3) top3_insert(top, cand_y[lane], cand_b[lane]);
+  warp_merge_top(top, zf);
+  EvalCtx ex;
+  ex.rk = rk; ex.row = row_ptr<DT>(p, row); ex.tau = tau; ex.slack_k = p.slack_scale; ex.grow = grow;
+  ex.ctr_lo = p.ctr_lo; ex.ctr_hi8 = p.ctr_hi8; ex.seg = 0; ex.V = (int)p.V;
+  float zt = 0.f;
+  const int id = sample_in_blocks<DT>(ex, top, lane, zt);
+  if (lane == 0) {
+    float logp = CUDART_NAN_F;
+    if (id >= 0) {
+      const double c = (double)__fdiv_rn(kLog2e, tau);
+      logp = (float)(((double)zt * c - (double)st.x) * kLn2 - log((double)st.y));
+    }
+    p.out_tok[row] = id;
+    if (p.out_logp) p.out_logp[row] = logp;
   }
 }
 
@@ -1889,13 +2079,15 @@ struct KernelSetup {
   int sms = 0;
 };
 
-template <int DT, int SAMPLER, bool RING>
+template <int DT, int SAMPLER>
 constexpr size_t dyn_smem_bytes() {
-  return (RING ? (size_t)kStages * kStageBytes : 0) + (SAMPLER == 0 ? (size_t)kStreamWarps * Fmt<DT>::kQueueBytes : 0) +
-         (SAMPLER == 1 ? (size_t)kStreamWarps * Fmt<DT>::kLB * 32 * sizeof(float) : 0);
+  return (size_t)kStreamWarps * RingStages<DT, SAMPLER>::value * kWarpBytes +
+         (SAMPLER == 0 ? (size_t)kStreamWarps * QueueBytes<DT>::value : 0) +
+         (SAMPLER == 1 ? (size_t)kStreamWarps * kRecordBytesPerWarp : 0);
 }
 
-template <int DT, int SAMPLER, bool RING>
+// Per device and kernel variant, once: opt in to the dynamic shared memory and ask how many CTAs fit an SM.
+template <int DT, int SAMPLER, bool GAP>
 cudaError_t setup_kernel(KernelSetup &out) {
   static std::mutex lock;
   static KernelSetup cache[64];
@@ -1905,8 +2097,8 @@ cudaError_t setup_kernel(KernelSetup &out) {
   if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
   std::lock_guard<std::mutex> hold(lock);
   if (cache[dev].ctas_per_sm == 0) {
-    auto kern = rows_kernel<DT, SAMPLER, RING>;
-    const size_t dyn = dyn_smem_bytes<DT, SAMPLER, RING>();
+    auto kern = rows_kernel<DT, SAMPLER, GAP>;
+    const size_t dyn = dyn_smem_bytes<DT, SAMPLER>();
     e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn);
     if (e != cudaSuccess) return e;
     KernelSetup ks;
@@ -1928,58 +2120,99 @@ unsigned long long next_call_id() {
   return (counter.fetch_add(1) + 1) & ((1ull << 48) - 1);
 }
 
-template <int DT, int SAMPLER, bool RING>
+// Test hook state (see arm_stall).
+std::atomic<long long> g_stall_tile{-1};
+std::atomic<unsigned long long> g_stall_wait_ns{0};
+
+constexpr unsigned long long kDefaultWaitNs = 2000000000ull;  // two seconds
+
+// Workspace: the pieces of cut rows first, then (sampler 1) per row a record for block_sample_kernel and per
+// tile the lanes' sums with their reference.
+size_t pieces_bytes() { return (size_t)kMaxGrid * 2 * kPieceBytes; }
+template <int DT>
+size_t partials_bytes(int64_t rows, int64_t V) {
+  const int64_t tiles = (V + Fmt<DT>::kWarpE - 1) / Fmt<DT>::kWarpE;
+  return (size_t)rows * 16 + (size_t)rows * tiles * (kRecordFloats * 4);
+}
+
+template <int DT, int SAMPLER, bool GAP>
 cudaError_t launch_one(RowsParams p, void *workspace, size_t workspace_bytes, cudaStream_t stream) {
   KernelSetup ks;
-  cudaError_t e = setup_kernel<DT, SAMPLER, RING>(ks);
+  cudaError_t e = setup_kernel<DT, SAMPLER, GAP>(ks);
   if (e != cudaSuccess) return e;
   int64_t slots = (int64_t)ks.sms * ks.ctas_per_sm;
   if (slots > kMaxGrid) slots = kMaxGrid;
-  p.tiles_per_row = (p.V + kTile - 1) / kTile;
+  p.tiles_per_row = (p.V + Fmt<DT>::kWarpE - 1) / Fmt<DT>::kWarpE;
   const int64_t tiles = p.rows * p.tiles_per_row;
   p.narrow = tiles < (int64_t(1) << 31) ? 1 : 0;
   if (tiles / slots >= (int64_t(1) << 30)) return cudaErrorInvalidValue;  // per-CTA tile counts are kept in 32 bits
-  const bool can_cut = workspace != nullptr && workspace_bytes >= rows_workspace_bytes();
-  // With a response mask the cost of a row is not known on the host: spread whole rows round-robin.
+  const bool can_cut = workspace != nullptr && workspace_bytes >= pieces_bytes();
+  if (SAMPLER == 1) {
+    if (!can_cut || workspace_bytes < pieces_bytes() + partials_bytes<DT>(p.rows, p.V)) return cudaErrorInvalidValue;
+    unsigned char *w = static_cast<unsigned char *>(workspace) + pieces_bytes();
+    p.ws_rowstat = reinterpret_cast<float4 *>(w);
+    w += (size_t)p.rows * 16;
+    p.ws_records = reinterpret_cast<float *>(w);
+  }
+  // With a response mask the cost of a row is not known on the host: with many rows, spread whole rows round-robin.
   p.interleaved = (!can_cut || (p.mask != nullptr && p.rows >= 4 * slots)) ? 1 : 0;
   int64_t grid = p.interleaved ? (p.rows < slots ? p.rows : slots) : (tiles < slots ? tiles : slots);
   p.tiles_q = tiles / grid;
   p.tiles_r = tiles % grid;
   p.ws_pieces = can_cut ? static_cast<unsigned char *>(workspace) : nullptr;
   p.call_id = next_call_id();
-  p.rehearse = 0;
+  p.wait_ns = kDefaultWaitNs;
+  p.stall_tile = g_stall_tile.exchange(-1);
+  if (p.stall_tile >= 0) p.wait_ns = g_stall_wait_ns.load();
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)grid);
   cfg.blockDim = dim3(kThreads);
-  cfg.dynamicSmemBytes = dyn_smem_bytes<DT, SAMPLER, RING>();
+  cfg.dynamicSmemBytes = dyn_smem_bytes<DT, SAMPLER>();
   cfg.stream = stream;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, rows_kernel<DT, SAMPLER, RING>, p);
+  e = cudaLaunchKernelEx(&cfg, rows_kernel<DT, SAMPLER, GAP>, p);
+  if (e != cudaSuccess || SAMPLER != 1) return e;
+  cfg.gridDim = dim3((unsigned)p.rows);
+  cfg.blockDim = dim3(kSampleWarps * 32);
+  cfg.dynamicSmemBytes = 0;
+  return cudaLaunchKernelEx(&cfg, block_sample_kernel<DT>, p);
+}
+
+template <int DT, int SAMPLER>
+cudaError_t launch_gap(const RowsParams &p, void *workspace, size_t workspace_bytes, cudaStream_t stream) {
+  return p.out_gap ? launch_one<DT, SAMPLER, true>(p, workspace, workspace_bytes, stream)
+                   : launch_one<DT, SAMPLER, false>(p, workspace, workspace_bytes, stream);
 }
 
 }  // namespace
 
-size_t rows_workspace_bytes() { return (size_t)kMaxGrid * 2 * kPieceBytes; }
+size_t rows_workspace_bytes() { return pieces_bytes(); }
+size_t sample_workspace_bytes(int dtype, int64_t rows, int64_t V) {
+  if (rows < 0 || V < 1) return pieces_bytes();
+  return pieces_bytes() + (dtype == 0 ? partials_bytes<0>(rows, V) : partials_bytes<1>(rows, V));
+}
+
+void arm_stall(int64_t stall_tile, unsigned long long wait_ns) {
+  g_stall_wait_ns.store(wait_ns);
+  g_stall_tile.store(stall_tile);
+}
 
 cudaError_t launch_rows(RowsParams p, int dtype, int sampler, bool aligned, void *workspace, size_t workspace_bytes,
                         cudaStream_t stream) {
-#define E3_DISPATCH(DT, SM)                                                                       \
-  return aligned ? launch_one<DT, SM, true>(p, workspace, workspace_bytes, stream)                \
-                 : launch_one<DT, SM, false>(p, workspace, workspace_bytes, stream)
+  p.bulk = aligned ? 1 : 0;
   if (dtype == 0) {
-    if (sampler < 0) { E3_DISPATCH(0, -1); }
-    if (sampler == 0) { E3_DISPATCH(0, 0); }
-    if (sampler == 1) { E3_DISPATCH(0, 1); }
-  } else {
-    if (sampler < 0) { E3_DISPATCH(1, -1); }
-    if (sampler == 0) { E3_DISPATCH(1, 0); }
-    if (sampler == 1) { E3_DISPATCH(1, 1); }
+    if (sampler < 0) return launch_gap<0, -1>(p, workspace, workspace_bytes, stream);
+    if (sampler == 0) return launch_gap<0, 0>(p, workspace, workspace_bytes, stream);
+    if (sampler == 1) return launch_gap<0, 1>(p, workspace, workspace_bytes, stream);
+  } else if (dtype == 1) {
+    if (sampler < 0) return launch_gap<1, -1>(p, workspace, workspace_bytes, stream);
+    if (sampler == 0) return launch_gap<1, 0>(p, workspace, workspace_bytes, stream);
+    if (sampler == 1) return launch_gap<1, 1>(p, workspace, workspace_bytes, stream);
   }
-#undef E3_DISPATCH
   return cudaErrorInvalidValue;
 }
 

@@ -35,11 +35,20 @@ __device__ __forceinline__ void block_reduce_2(double &a, double &b, double *sh 
   }
 }
 
+// Both stages may be launched with programmatic stream serialization behind the kernel that writes `ent`:
+// they wait for it (and for its writes) before they touch memory.  Without that launch attribute the wait
+// returns at once.
+__device__ __forceinline__ void wait_for_stream_predecessor() {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
 // Stage 1: block b sums tokens [b*chunk, (b+1)*chunk) in a fixed order and stores one partial.
 __global__ void __launch_bounds__(kMeanThreads) mean_partial_kernel(const float *__restrict__ ent,
                                                                     const uint8_t *__restrict__ mask, int64_t n,
                                                                     int64_t chunk, MeanPartial *__restrict__ part) {
   __shared__ double sh[2 * kMeanThreads / 32];
+  wait_for_stream_predecessor();
   const int64_t lo = (int64_t)blockIdx.x * chunk;
   const int64_t hi = lo + chunk < n ? lo + chunk : n;
   double s = 0.0, c = 0.0;
@@ -51,16 +60,17 @@ __global__ void __launch_bounds__(kMeanThreads) mean_partial_kernel(const float 
   if (threadIdx.x == 0) { part[blockIdx.x].sum = s; part[blockIdx.x].cnt = c; }
 }
 
-// Stage 2: one block adds the partials in index order and writes mean and count.
+// Stage 2: one block adds the partials in index order and writes mean (or, with want_sum, the sum) and count.
 __global__ void __launch_bounds__(kMeanThreads) mean_final_kernel(const MeanPartial *__restrict__ part, int nparts,
                                                                   double *__restrict__ out_mean,
-                                                                  double *__restrict__ out_count) {
+                                                                  double *__restrict__ out_count, int want_sum) {
   __shared__ double sh[2 * kMeanThreads / 32];
+  wait_for_stream_predecessor();
   double s = 0.0, c = 0.0;
   for (int j = threadIdx.x; j < nparts; j += kMeanThreads) { s += part[j].sum; c += part[j].cnt; }
   block_reduce_2(s, c, sh);
   if (threadIdx.x == 0) {
-    *out_mean = c > 0.0 ? s / c : CUDART_NAN;
+    *out_mean = want_sum ? s : (c > 0.0 ? s / c : CUDART_NAN);
     *out_count = c;
   }
 }
@@ -101,7 +111,8 @@ __global__ void __launch_bounds__(256) group_advantage_kernel(const float *__res
   for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
   const double denom = unbiased ? (double)(n - 1) : (double)n;
   const double sd = n == 1 ? 0.0 : sqrt(ss / denom);
-  const double inv = 1.0 / (sd + (double)eps);
+  // std + eps == 0 (eps == 0 and identical rewards): every r_i - mean is 0 and the advantage is 0, not 0/0
+  const double inv = sd + (double)eps > 0.0 ? 1.0 / (sd + (double)eps) : 0.0;
   for (int64_t i = lo + lane; i < hi; i += 32)
     adv[i] = n == 1 ? 0.f : (float)(((double)rewards[i] - mean) * inv);
   if (flags && lane == 0) flags[g] = (uint8_t)((differs ? 0 : 1) | (nonzero ? 0 : 2));
@@ -119,13 +130,24 @@ int mean_blocks(int64_t n) {
 size_t mean_workspace_bytes(int64_t n) { return (size_t)mean_blocks(n) * sizeof(MeanPartial); }
 
 cudaError_t launch_masked_mean(const float *ent, const uint8_t *mask, int64_t n, double *out_mean,
-                               double *out_count, void *workspace, cudaStream_t stream) {
+                               double *out_count, void *workspace, bool want_sum, cudaStream_t stream) {
   const int blocks = mean_blocks(n);
   const int64_t chunk = (n + blocks - 1) / blocks;
   MeanPartial *part = static_cast<MeanPartial *>(workspace);
-  mean_partial_kernel<<<blocks, kMeanThreads, 0, stream>>>(ent, mask, n, chunk, part);
-  mean_final_kernel<<<1, kMeanThreads, 0, stream>>>(part, blocks, out_mean, out_count);
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg = {};
+  cfg.blockDim = dim3(kMeanThreads);
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  cfg.gridDim = dim3((unsigned)blocks);
+  cudaError_t e = cudaLaunchKernelEx(&cfg, mean_partial_kernel, ent, mask, n, chunk, part);
+  if (e != cudaSuccess) return e;
+  cfg.gridDim = dim3(1);
+  return cudaLaunchKernelEx(&cfg, mean_final_kernel, (const MeanPartial *)part, blocks, out_mean, out_count,
+                            want_sum ? 1 : 0);
 }
 
 cudaError_t launch_group_advantage(const float *rewards, const int64_t *off, int64_t n_groups, float eps,

@@ -34,7 +34,9 @@ def test_library_exports_every_declared_symbol(e3):
 def test_status_strings_and_workspace(e3):
     assert e3.status_string(0) == "E3_OK"
     assert e3.status_string(5) == "E3_ERR_INFEASIBLE"
-    assert e3.e3_workspace_bytes(e3.E3_CALL_SAMPLE, 512, 151936, e3.E3_BF16) >= 1024 * 136
+    assert e3.e3_workspace_bytes(e3.E3_CALL_SAMPLE, 512, 151936, e3.E3_BF16) >= 1024 * 256 + 512 * 75 * 132 + 512 * 16
+    assert e3.e3_workspace_bytes(e3.E3_CALL_SAMPLE, 512, 151936, e3.E3_BF16) < 16 * 512 * 151936 * 2 // 256
+    assert e3.e3_workspace_bytes(e3.E3_CALL_TOKEN_LOGP_ENTROPY, 131072, 151936, e3.E3_BF16) >= 1024 * 256 + 16
     assert e3.e3_workspace_bytes(e3.E3_CALL_MASKED_MEAN_ENTROPY, 131072) >= 16
     assert e3.e3_workspace_bytes(e3.E3_CALL_MASKED_MEAN_ENTROPY, 0) >= 16
 
@@ -42,21 +44,46 @@ def test_status_strings_and_workspace(e3):
 def test_device_calls_reject_bad_arguments_on_the_host(e3):
     L = e3.lib()
     # checked before any CUDA call is made, so these run without a device
-    assert L.e3_sample(None, 7, 1, 8, 8, None, 0, 0, 0, 0, None, None, None, None, 0, None) == 2   # dtype
-    assert L.e3_sample(None, 0, -1, 8, 8, None, 0, 0, 0, 0, None, None, None, None, 0, None) == 1  # rows < 0
-    assert L.e3_sample(None, 0, 1, 8, 4, None, 0, 0, 0, 0, None, None, None, None, 0, None) == 1   # stride < V
-    assert L.e3_sample(None, 0, 1, 1 << 31, 1 << 31, None, 0, 0, 0, 0, None, None, None, None, 0, None) == 1
-    assert L.e3_sample(None, 0, 0, 8, 8, None, 0, 0, 0, 0, None, None, None, None, 0, None) == 0   # rows == 0
-    assert L.e3_sample(None, 0, 0, 8, 8, None, 0, 1 << 56, 0, 0, None, None, None, None, 0, None) == 1
-    assert L.e3_sample(None, 0, 0, 8, 8, None, 0, 0, 0, 3, None, None, None, None, 0, None) == 1   # sampler
-    assert L.e3_sample(1024, 0, 1, 8, 8, None, 0, 0, 0, 0, None, None, None, None, 0, None) == 1   # temps NULL
-    assert L.e3_sample(1026, 0, 1, 8, 8, 1024, 0, 0, 0, 0, 1024, None, None, None, 0, None) == 3   # misaligned
-    assert L.e3_token_logp_entropy(None, 0, 0, 8, 8, None, None, None, 1.0, None, None, None, 0, None) == 0
-    assert L.e3_token_logp_entropy(1024, 0, 1, 8, 8, None, None, None, 1.0, None, None, None, 0, None) == 1
+    def sample(logits, dt, rows, V, stride, temps=None, counter=0, row_base=0, sampler=0, out_tok=None,
+               ws=None, ws_bytes=0):
+        return L.e3_sample(logits, dt, rows, V, stride, temps, 0, counter, row_base, sampler, out_tok, None, None,
+                           None, None, ws, ws_bytes, None)
+
+    def token(logits, dt, rows, V, stride, targets=None, out_ent=None, out_sum=None, out_count=None, ws=None,
+              ws_bytes=0):
+        return L.e3_token_logp_entropy(logits, dt, rows, V, stride, targets, None, None, 1.0, None, out_ent, None,
+                                       out_sum, out_count, None, ws, ws_bytes, None)
+
+    assert sample(None, 7, 1, 8, 8) == 2                      # dtype
+    assert sample(None, 0, -1, 8, 8) == 1                     # rows < 0
+    assert sample(None, 0, 1, 8, 4) == 1                      # stride < V
+    assert sample(None, 0, 1, 1 << 31, 1 << 31) == 1          # V too large
+    assert sample(None, 0, 0, 8, 8) == 0                      # rows == 0
+    assert sample(None, 0, 0, 8, 8, counter=1 << 56) == 1
+    assert sample(None, 0, 0, 8, 8, sampler=3) == 1           # sampler
+    assert sample(1024, 0, 1, 8, 8) == 1                      # temps NULL
+    assert sample(1026, 0, 1, 8, 8, temps=1024, out_tok=1024) == 3   # misaligned
+    # the row number is one 32-bit word of the Philox counter
+    assert sample(None, 0, 0, 8, 8, row_base=-1) == 1
+    assert sample(None, 0, 0, 8, 8, row_base=1 << 32) == 0            # no rows: nothing exceeds the range
+    assert sample(1024, 0, 1, 8, 8, temps=1024, out_tok=1024, row_base=1 << 32) == 1
+    assert sample(1024, 0, 2, 8, 8, temps=1024, out_tok=1024, row_base=(1 << 32) - 1) == 1
+    # the blocked sampler needs its workspace
+    assert sample(1024, 0, 1, 8, 8, temps=1024, out_tok=1024, sampler=1) == 4
+    assert sample(1024, 0, 1, 8, 8, temps=1024, out_tok=1024, sampler=1, ws=4096, ws_bytes=1 << 18) == 4
+    assert token(None, 0, 0, 8, 8) == 0
+    assert token(1024, 0, 1, 8, 8) == 1                       # targets NULL
+    # fused mean entropy: both scalars or none, needs out_ent and the workspace
+    assert token(1024, 0, 1, 8, 8, targets=1024, out_ent=1024, out_sum=2048) == 1
+    assert token(1024, 0, 1, 8, 8, targets=1024, out_sum=2048, out_count=2056) == 1
+    assert token(1024, 0, 1, 8, 8, targets=1024, out_ent=1024, out_sum=2048, out_count=2056) == 4
+    assert token(1024, 0, 1, 8, 8, targets=1024, out_ent=1024, out_sum=2052, out_count=2056) == 3
     assert L.e3_masked_mean_entropy(None, None, -1, None, None, None, 0, None) == 1
     assert L.e3_masked_mean_entropy(1024, None, 4, 1024, 1032, None, 0, None) == 4                  # workspace
     assert L.e3_group_advantage(None, None, 0, 1e-6, 1, None, None, None) == 0
     assert L.e3_group_advantage(None, None, 2, 1e-6, 1, None, None, None) == 1
+    assert L.e3_group_advantage(None, None, 2, -1.0, 1, None, None, None) == 1                       # eps < 0
+    assert L.e3_group_advantage(None, None, 2, float("inf"), 1, None, None, None) == 1
     with pytest.raises(ValueError):
         import torch
         e3.e3_sample(torch.zeros(2, 8), torch.ones(2), 0, 0)   # CPU tensors: there is no CPU path
