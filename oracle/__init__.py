@@ -145,6 +145,19 @@ def token_logp_entropy(logits: np.ndarray, targets: np.ndarray, mask=None, temps
     return tuple(outs)
 
 
+def row_gap(logits: np.ndarray, temps=None, temp_scalar: float = 1.0, mask=None, greedy: bool = False) -> np.ndarray:
+    """Mean logit gap beta * sum_i p_i (z_max - z_i) per row, float64 [rows]."""
+    ptr, dt, rows, V, stride = _logits_args(logits)
+    mask = None if mask is None else np.ascontiguousarray(mask, dtype=np.uint8)
+    temps = None if temps is None else np.ascontiguousarray(temps, dtype=np.float32)
+    out = np.empty(rows, np.float64)
+    rc = lib().e3o_row_gap(ptr, dt, C.c_int64(rows), C.c_int64(V), C.c_int64(stride), _p(mask), _p(temps),
+                           C.c_float(temp_scalar), C.c_int(int(greedy)), _p(out))
+    if rc != 0:
+        raise ValueError("e3o_row_gap: invalid argument")
+    return out
+
+
 def token_logp_entropy_backward(logits: np.ndarray, targets: np.ndarray, g_logp=None, g_ent=None, mask=None, temps=None,
                                 temp_scalar: float = 1.0) -> np.ndarray:
     """Gradient with respect to the logits, float64 [rows, V]."""

@@ -362,6 +362,51 @@ int e3o_token_logp_entropy(const void *logits, int dt, int64_t rows, int64_t V, 
 }
 
 /* ------------------------------------------------------------------------- */
+/* Mean logit gap of a row in units of tau (App. A): with Delta_i = z_max -   */
+/* z_i and beta = 1/tau,  gap = beta sum_i p_i Delta_i = sum_i p_i (s_max -   */
+/* s_i), the first term of the decomposition H = beta sum p Delta + ln Z.     */
+/* It is the quantity Eq. "tp_relation_1" needs an estimate of (beta Delta of */
+/* the two-level model).  Rows with mask == 0 give 0; tau == 0 with greedy    */
+/* != 0 gives 0 (point mass on the arg-max); an invalid row gives NaN.        */
+/* Written out from the definition with its own loops (no shared state with   */
+/* the entropy routine above).                                                */
+/* Pins: two-level row -> beta Delta q / (1 + q), q = (N-1) exp(-beta Delta); */
+/* uniform row -> 0; H = ln Z + gap with H from -sum p ln p; invariance under */
+/* a shift of the row.                                                        */
+/* ------------------------------------------------------------------------- */
+int e3o_row_gap(const void *logits, int dt, int64_t rows, int64_t V, int64_t row_stride, const uint8_t *mask,
+                const float *temps, float temp_scalar, int greedy, double *out_gap) {
+  if (rows < 0 || V < 1 || row_stride < V || (dt != E3O_F32 && dt != E3O_BF16) || !out_gap) return 1;
+  size_t esz = dt == E3O_F32 ? 4 : 2;
+#pragma omp parallel for schedule(dynamic, 1)
+  for (int64_t r = 0; r < rows; ++r) {
+    if (mask && !mask[r]) { out_gap[r] = 0.0; continue; }
+    const char *row = (const char *)logits + (size_t)r * (size_t)row_stride * esz;
+    double tau = temps ? (double)temps[r] : (double)temp_scalar;
+    int bad = 0;
+    double zmax = -INFINITY;
+    for (int64_t i = 0; i < V; ++i) {
+      double z = widen(row, dt, i);
+      if (isnan(z) || z == INFINITY) bad = 1;
+      if (z > zmax) zmax = z;
+    }
+    if (bad || zmax == -INFINITY) { out_gap[r] = NAN; continue; }
+    if (greedy && tau == 0.0) { out_gap[r] = 0.0; continue; }
+    if (!(tau > 0.0) || isinf(tau)) { out_gap[r] = NAN; continue; }
+    double beta = 1.0 / tau, Z = 0.0, num = 0.0;
+    for (int64_t i = 0; i < V; ++i) {
+      double delta = zmax - widen(row, dt, i); /* Delta_i >= 0, +inf for a -inf logit */
+      if (delta == INFINITY) continue;          /* p_i = 0 */
+      double w = exp(-beta * delta);
+      Z += w;
+      num += w * (beta * delta);
+    }
+    out_gap[r] = num / Z;
+  }
+  return 0;
+}
+
+/* ------------------------------------------------------------------------- */
 /* Gradient of the training-side outputs with respect to the logits.  The     */
 /* objective of Sec. 3.1 depends on the logits through ln pi(o_t), the        */
 /* entropy-regularised objective discussed in Sec. 4.2 also through H; with   */
@@ -461,7 +506,8 @@ int e3o_group_advantage(const float *rewards, const int64_t *group_offsets, int6
     double denom = unbiased ? (double)(n - 1) : (double)n;
     double sd = (n == 1) ? 0.0 : sqrt(ss / denom);
     for (int64_t i = lo; i < hi; ++i)
-      out_adv[i] = (n == 1) ? 0.0 : ((double)rewards[i] - mean) / (sd + (double)eps);
+      /* Sec. 4.2: a group whose rewards are all equal has advantage 0; with eps == 0 the quotient would be 0/0 */
+      out_adv[i] = (n == 1 || sd + (double)eps == 0.0) ? 0.0 : ((double)rewards[i] - mean) / (sd + (double)eps);
     if (out_flags) out_flags[g] = (uint8_t)((all_equal ? 1 : 0) | (all_zero ? 2 : 0));
   }
   return 0;

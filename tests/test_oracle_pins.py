@@ -385,6 +385,68 @@ def test_masked_mean_entropy():
 
 
 # ----------------------------------------------------------------------------------------------
+# Mean logit gap (App. A: beta sum p_i Delta_i, the first term of H = beta sum p Delta + ln Z)
+# ----------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("N,delta,tau", [(151936, 12.0, 1.0), (151936, 25.0, 1.0), (256000, 25.0, 2.0), (1000, 3.0, 0.5),
+                                          (32000, 6.0, 0.7)])
+def test_row_gap_two_level_closed_form(N, delta, tau):
+    """One logit at +Delta, N-1 at 0: gap = beta Delta q / (1 + q) with q = (N-1) e^{-beta Delta}."""
+    z = np.zeros((1, N), np.float32)
+    z[0, N // 5] = delta
+    beta = 1.0 / float(np.float32(tau))
+    q = (N - 1) * math.exp(-beta * delta)
+    gap = oracle.row_gap(z, temp_scalar=tau)
+    assert gap[0] == pytest.approx(beta * delta * q / (1.0 + q), rel=1e-10, abs=1e-12)
+
+
+def test_row_gap_special_cases_and_entropy_identity():
+    rng = np.random.default_rng(21)
+    V = 5003
+    z = (3.0 * rng.normal(size=(6, V))).astype(np.float32)
+    z[1, 17:900] = -np.inf                       # entries without mass
+    temps = np.array([0.6, 1.0, 1.4, 0.3, 2.0, 1.0], np.float32)
+    gap = oracle.row_gap(z, temps=temps)
+    # H from -sum p ln p (its own routine) equals ln Z + gap, with ln Z from a library log-sum-exp
+    _, ent, _ = oracle.token_logp_entropy(z, np.zeros(6, np.int32), temps=temps)
+    for r in range(6):
+        s = z[r].astype(np.float64) / float(temps[r])
+        lnZ = scipy.special.logsumexp(s - s.max())
+        assert ent[r] == pytest.approx(lnZ + gap[r], rel=1e-11, abs=1e-11)
+        # the gap is the softmax-weighted mean of s_max - s_i: a library softmax gives the same
+        p = scipy.special.softmax(s)
+        keep = np.isfinite(s)
+        assert gap[r] == pytest.approx(float(np.sum(p[keep] * (s.max() - s[keep]))), rel=1e-11, abs=1e-12)
+    # shifting a row changes nothing (multiples of 1/8: adding 32 is exact)
+    zs = np.round(z[:1] * 8) / 8
+    assert oracle.row_gap(zs + np.float32(32.0), temp_scalar=1.0)[0] == pytest.approx(oracle.row_gap(zs, temp_scalar=1.0)[0], rel=1e-12)
+    # a uniform row has no gap; a single entry has none either
+    assert oracle.row_gap(np.full((1, 777), -2.5, np.float32), temp_scalar=0.7)[0] == 0.0
+    assert oracle.row_gap(np.array([[4.0]], np.float32), temp_scalar=0.7)[0] == 0.0
+    # two entries at distance d: gap = beta d e^{-beta d} / (1 + e^{-beta d})
+    d, tau = 1.5, 0.5
+    g2 = oracle.row_gap(np.array([[0.25, 0.25 - d]], np.float32), temp_scalar=tau)[0]
+    assert g2 == pytest.approx((d / tau) * math.exp(-d / tau) / (1.0 + math.exp(-d / tau)), rel=1e-13)
+    # masked rows give 0; greedy rows (tau == 0 where the caller allows it) give 0; bad rows NaN
+    zz = np.array([[0.0, 1.0, 2.0], [0.0, np.nan, 1.0], [np.inf, 0.0, 0.0], [-np.inf, -np.inf, -np.inf], [0.0, 1.0, 2.0]], np.float32)
+    g = oracle.row_gap(zz, temps=np.array([1.0, 1.0, 1.0, 1.0, 0.0], np.float32), mask=np.array([0, 1, 1, 1, 1], np.uint8), greedy=True)
+    assert g[0] == 0.0 and np.isnan(g[1]) and np.isnan(g[2]) and np.isnan(g[3]) and g[4] == 0.0
+    g = oracle.row_gap(zz[4:], temps=np.array([0.0], np.float32), greedy=False)
+    assert np.isnan(g[0])
+    assert np.isnan(oracle.row_gap(zz[:1], temp_scalar=-1.0)[0])
+
+
+def test_row_gap_estimates_the_gap_of_the_two_level_model():
+    """Eq. "tp_relation_1" wants Delta / tau_0 of the two-level model; for such a row in the small-entropy regime the
+    measured gap statistic divided by the mass off the leader, (gap / (1 - p_max)), is exactly beta Delta."""
+    N, delta, tau = 151936, 20.0, 1.25
+    z = np.zeros((1, N), np.float32)
+    z[0, 3] = delta
+    gap = oracle.row_gap(z, temp_scalar=tau)[0]
+    lp, _, _ = oracle.token_logp_entropy(z, np.array([3]), temp_scalar=tau)
+    assert gap / (1.0 - math.exp(lp[0])) == pytest.approx(delta / tau, rel=1e-9)
+
+
+# ----------------------------------------------------------------------------------------------
 # Group advantage (Eq. "adv")
 # ----------------------------------------------------------------------------------------------
 def test_group_advantage_worked_example():
@@ -425,6 +487,10 @@ def test_group_advantage_matches_textbook_zscore_and_invariants():
     a1, _ = oracle.group_advantage(np.array([0, 1], np.float32), [0, 2], eps=0.5)
     sd = math.sqrt(0.5)
     assert a0[1] == pytest.approx(0.5 / sd) and a1[1] == pytest.approx(0.5 / (sd + 0.5))
+    # identical rewards give exactly zero also without eps (Sec. 4.2: such groups carry no signal), never 0/0
+    for unbiased in (True, False):
+        az, fz = oracle.group_advantage(np.array([1, 1, 1, 0.5, 0.5], np.float32), [0, 3, 5], eps=0.0, unbiased=unbiased)
+        assert np.all(az == 0.0) and fz.tolist() == [1, 1]
 
 
 # ----------------------------------------------------------------------------------------------
