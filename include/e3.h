@@ -369,6 +369,16 @@ E3_API double e3_anneal_target(const e3_sched *s);
  */
 E3_API void e3_test_arm_stall(int64_t tile, uint64_t wait_ns);
 
+/*
+ * Measurement aid: reads `bytes` (a multiple of 16) of device memory at `buf` (16-byte aligned) once, with a
+ * plain grid of four thread blocks per SM that only adds the words up -- the practical read-only ceiling
+ * of the device, against which the benchmark reports the row kernels.  `scratch`: device memory of at least
+ * 8 bytes per thread block (E3_PROBE_SCRATCH_BYTES covers every device), receives one checksum per block.
+ * E3_ERR_INVALID_ARG for NULL or misaligned arguments, E3_ERR_WORKSPACE for a scratch that is too small.
+ */
+#define E3_PROBE_SCRATCH_BYTES 65536
+E3_API e3_status e3_probe_read(const void *buf, size_t bytes, void *scratch, size_t scratch_bytes, void *stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -27,7 +27,7 @@ EXPORTS = ("e3_status_string", "e3_workspace_bytes", "e3_sample", "e3_token_logp
            "e3_token_logp_entropy_backward", "e3_grpo_objective",
            "e3_masked_mean_entropy", "e3_masked_mean_entropy_static", "e3_group_advantage", "e3_allocate_budget", "e3_update_temperature",
            "e3_anneal_target", "e3_entropy_gap", "e3_update_temperature_gap", "e3_difficulty_accumulate", "e3_difficulty_rank", "e3_budget_curriculum",
-           "e3_test_arm_stall")
+           "e3_test_arm_stall", "e3_probe_read")
 
 
 class E3Error(RuntimeError):
@@ -100,6 +100,8 @@ def lib() -> C.CDLL:
                                            C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
         L.e3_anneal_target.restype = C.c_double
         L.e3_anneal_target.argtypes = [C.POINTER(e3_sched)]
+        L.e3_probe_read.restype = C.c_int
+        L.e3_probe_read.argtypes = [C.c_void_p, C.c_size_t, C.c_void_p, C.c_size_t, C.c_void_p]
         L.e3_test_arm_stall.restype = None
         L.e3_test_arm_stall.argtypes = [C.c_int64, C.c_uint64]
         _lib = L
@@ -430,3 +432,17 @@ def e3_budget_curriculum(G: int, step: int, G_min_limit: int, G_max_limit: int, 
 def e3_test_arm_stall(tile: int, wait_ns: int) -> None:
     """Test hook: the next row call leaves one 4 KiB tile uncopied and bounds its waits by ``wait_ns``."""
     lib().e3_test_arm_stall(int(tile), int(wait_ns))
+
+
+E3_PROBE_SCRATCH_BYTES = 65536
+
+
+def e3_probe_read(buf, scratch=None, stream=None):
+    """Measurement aid: one read-only pass over ``buf`` (a CUDA tensor whose size is a multiple of 16 bytes)."""
+    _dev(buf, "buf")
+    if scratch is None:
+        scratch = torch.empty(E3_PROBE_SCRATCH_BYTES, dtype=torch.uint8, device=buf.device)
+    st = lib().e3_probe_read(_ptr(buf), buf.numel() * buf.element_size(), _ptr(scratch),
+                             scratch.numel() * scratch.element_size(), _stream(stream))
+    _check("e3_probe_read", st)
+    return scratch

@@ -67,6 +67,7 @@ def test_config1_tiny_sampling_step(e3, sampler):
     logits = inputs.zipf_gaussian_logits(rows, V, seed=1, dtype=torch.float32, device=DEV)
     temps = inputs.uniform_temps(rows, seed=2, device=DEV)
     info = _check_sample(e3, logits, temps, seed=0, counter=0, sampler=sampler, name="c1")
+    print("parity:", {"case": f"c1.s{sampler}", "rows_checked": rows, **info})
     assert info["mismatch_near_tie"] == 0
     sizes = [8] * 8
     rewards = inputs.bernoulli_rewards(sizes, 0.5, seed=3, device=DEV)
