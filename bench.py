@@ -49,8 +49,8 @@ GROUP = 8
 METRIC = "logit rows/s, fused sample+entropy, V=151,936"
 UNIT = "rows/s"
 # dram__bytes_read.sum + dram__bytes_write.sum of one e3_sample launch of this workload (ncu capture summarised in
-# profiles/rows_kernel_c2_ncu_full.txt); only for the kernel variant that was captured.
-NCU_TRAFFIC_BYTES = {1: 160.7e6}
+# profiles/rows_kernel_c2_ncu_full.txt and rows_kernel_sampler0_c2_ncu_full.txt), streaming kernel only.
+NCU_TRAFFIC_BYTES = {0: 161.7e6, 1: 160.2e6}
 WORKLOAD = "rollout decode step: 512 rows (64 prompts x 8 rollouts) x V=151,936 bf16, 256 decode steps"
 
 
@@ -291,6 +291,8 @@ def main():
     ap.add_argument("--impl", default="e3", choices=["e3", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-configs", action="store_true",
+                    help="skip the other configurations (c1, c3, c4, c5): a short run, e.g. for a launch list")
     ap.add_argument("--profile-launches", type=int, default=0,
                     help="run this many decode launches plus one training-side launch and exit (for ncu captures)")
     args = ap.parse_args()
@@ -369,6 +371,8 @@ def main():
         for d in range(args.profile_launches):
             e3.e3_sample(ring[d % RING], temps, 0, d, row_base, args.sampler, out_tok=toks[d % RING],
                          out_logp=logp, out_ent=ent)
+        for d in range(2):   # the training-side kernel on one ring buffer (512 rows), then on the whole batch
+            e3.e3_token_logp_entropy(ring[d], all_toks[:ROWS], temps=temps, out_logp=logp, out_ent=ent)
         e3.e3_token_logp_entropy(batch, all_toks, mask=mask, temp_scalar=1.0, out_logp=t_logp, out_ent=t_ent)
         dz = torch.empty((ROWS, V), dtype=torch.bfloat16, device=dev)
         e3.e3_token_logp_entropy_backward(batch[:ROWS], all_toks[:ROWS], t_logp[:ROWS], t_ent[:ROWS], t_logp[:ROWS],
@@ -501,7 +505,8 @@ def main():
     configs, parity = None, None
     if rank == 0 and world == 1:
         peak_gbs, _ = _peaks()
-        configs = other_configs(e3, inputs, dev, peak_gbs, time_alone)
+        if not args.no_configs:
+            configs = other_configs(e3, inputs, dev, peak_gbs, time_alone)
         if not args.no_cpu_baseline:
             parity = verified_step(e3, inputs, ring[0], temps, toks[0], logp, ent, args.sampler)
 
