@@ -88,7 +88,8 @@ typedef enum {
   E3_CALL_SAMPLE = 0,
   E3_CALL_TOKEN_LOGP_ENTROPY = 1,
   E3_CALL_MASKED_MEAN_ENTROPY = 2,
-  E3_CALL_GRPO_OBJECTIVE = 3
+  E3_CALL_GRPO_OBJECTIVE = 3,
+  E3_CALL_SEQUENCE_MEAN_ENTROPY = 4
 } e3_call;
 
 /* Human-readable name of a status code (static string). */
@@ -96,7 +97,7 @@ E3_API const char *e3_status_string(e3_status s);
 
 /* Bytes of device scratch a call uses for the given problem size.  For
  * E3_CALL_MASKED_MEAN_ENTROPY `rows` is the number of tokens n, for E3_CALL_GRPO_OBJECTIVE the number of
- * responses n_seq; V, dt are ignored for both.  E3_CALL_SAMPLE: 256 KiB for the partial states of cut rows plus,
+ * responses n_seq, for E3_CALL_SEQUENCE_MEAN_ENTROPY the number of sequences n_seq; V, dt are ignored for these.  E3_CALL_SAMPLE: 256 KiB for the partial states of cut rows plus,
  * for E3_SAMPLER_BLOCK, the per-lane sums the second kernel reads (about 1/32 of the bytes of the logits);
  * E3_CALL_TOKEN_LOGP_ENTROPY: 256 KiB plus the partial sums of the fused mean entropy.
  * Scratch contents on entry never matter.  A workspace must not be shared by calls that can run
@@ -208,6 +209,20 @@ E3_API e3_status e3_token_logp_entropy_backward(const void *logits, e3_dtype dt,
 E3_API e3_status e3_masked_mean_entropy(const float *ent, const uint8_t *mask, int64_t n,
                                  double *out_mean, double *out_count,
                                  void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * The other reading of "average entropy" (Sec. 4.2 does not say which): the mean over sequences of each
+ * sequence's mean token entropy.  Tokens are laid out [n_seq, seq_len]; mask marks the response tokens.
+ *   out_mean  = (1 / S) sum_s ( sum_t mask[s,t] ent[s,t] / sum_t mask[s,t] ), over the S sequences that have a token
+ *   out_count = S.   S == 0 gives mean NaN.
+ * Long responses weigh as much as short ones here, while e3_masked_mean_entropy weighs every token equally.
+ * fp64, fixed order (one thread block per sequence, then one block over the sequences in index order).
+ *   ent, mask   device float / uint8 [n_seq * seq_len], mask may be NULL (= all ones);  n_seq < 2^31
+ *   workspace   e3_workspace_bytes(E3_CALL_SEQUENCE_MEAN_ENTROPY, n_seq, 0, 0) bytes of device scratch, 8-byte aligned
+ */
+E3_API e3_status e3_sequence_mean_entropy(const float *ent, const uint8_t *mask, int64_t n_seq, int64_t seq_len,
+                                          double *out_mean, double *out_count,
+                                          void *workspace, size_t workspace_bytes, void *stream);
 
 /*
  * The same mean entropy for callers that have no scratch memory to give.  (The paper has no

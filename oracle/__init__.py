@@ -187,6 +187,19 @@ def masked_mean_entropy(ent: np.ndarray, mask=None):
     return mean.value, cnt.value
 
 
+def sequence_mean_entropy(ent: np.ndarray, mask=None):
+    """Mean over sequences of the per-sequence mean entropy; ent [n_seq, seq_len].  Returns (mean, sequences used)."""
+    ent = np.ascontiguousarray(ent, dtype=np.float32)
+    assert ent.ndim == 2
+    mask = None if mask is None else np.ascontiguousarray(mask, dtype=np.uint8)
+    mean, cnt = C.c_double(), C.c_double()
+    rc = lib().e3o_sequence_mean_entropy(_p(ent), _p(mask), C.c_int64(ent.shape[0]), C.c_int64(ent.shape[1]),
+                                         C.byref(mean), C.byref(cnt))
+    if rc != 0:
+        raise ValueError("e3o_sequence_mean_entropy: invalid argument")
+    return mean.value, cnt.value
+
+
 def group_advantage(rewards: np.ndarray, group_offsets: np.ndarray, eps: float = 1e-6, unbiased: bool = True):
     """Returns (adv float64 [n], flags uint8 [n_groups])."""
     rewards = np.ascontiguousarray(rewards, dtype=np.float32)

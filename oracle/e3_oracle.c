@@ -485,6 +485,26 @@ int e3o_masked_mean_entropy(const float *ent, const uint8_t *mask, int64_t n, do
 /* of one gets 0.  flags: bit 0 = all rewards equal, bit 1 = all rewards 0.   */
 /* Pins: worked example r=(1,0,...,0); zero group mean; textbook z-score.     */
 /* ------------------------------------------------------------------------- */
+/* The other reading of "average entropy" (Sec. 4.2): the mean over sequences of every sequence's own mean   */
+/* token entropy; tokens laid out [n_seq, seq_len]; sequences without a token take no part; none at all: NaN. */
+/* Pins: brute force; equal-length sequences give the token mean; hand case where the two readings differ.    */
+int e3o_sequence_mean_entropy(const float *ent, const uint8_t *mask, int64_t n_seq, int64_t seq_len,
+                              double *out_mean, double *out_count) {
+  if (n_seq < 0 || seq_len < 0 || !out_mean || !out_count) return 1;
+  double total = 0.0, used = 0.0;
+  for (int64_t s = 0; s < n_seq; ++s) {
+    double sum = 0.0, cnt = 0.0;
+    for (int64_t t = 0; t < seq_len; ++t) {
+      int64_t j = s * seq_len + t;
+      if (!mask || mask[j]) { sum += (double)ent[j]; cnt += 1.0; }
+    }
+    if (cnt > 0.0) { total += sum / cnt; used += 1.0; }
+  }
+  *out_mean = used > 0.0 ? total / used : NAN;
+  *out_count = used;
+  return 0;
+}
+
 int e3o_group_advantage(const float *rewards, const int64_t *group_offsets, int64_t n_groups, float eps,
                         int unbiased, double *out_adv, uint8_t *out_flags) {
   if (n_groups < 0) return 1;

@@ -21,13 +21,14 @@ E3_STATUS_TIMEOUT = 1
 E3_F32, E3_BF16 = 0, 1
 E3_SAMPLER_TOKEN, E3_SAMPLER_BLOCK, E3_SAMPLER_TOKEN_AUDIT = 0, 1, 2
 E3_CALL_SAMPLE, E3_CALL_TOKEN_LOGP_ENTROPY, E3_CALL_MASKED_MEAN_ENTROPY, E3_CALL_GRPO_OBJECTIVE = 0, 1, 2, 3
+E3_CALL_SEQUENCE_MEAN_ENTROPY = 4
 E3_SAMPLE_BLOCK = 256
 
 EXPORTS = ("e3_status_string", "e3_workspace_bytes", "e3_sample", "e3_token_logp_entropy",
            "e3_token_logp_entropy_backward", "e3_grpo_objective",
            "e3_masked_mean_entropy", "e3_masked_mean_entropy_static", "e3_group_advantage", "e3_allocate_budget", "e3_update_temperature",
            "e3_anneal_target", "e3_entropy_gap", "e3_update_temperature_gap", "e3_difficulty_accumulate", "e3_difficulty_rank", "e3_budget_curriculum",
-           "e3_test_arm_stall", "e3_probe_read")
+           "e3_test_arm_stall", "e3_probe_read", "e3_sequence_mean_entropy")
 
 
 class E3Error(RuntimeError):
@@ -72,6 +73,9 @@ def lib() -> C.CDLL:
         L.e3_masked_mean_entropy.restype = C.c_int
         L.e3_masked_mean_entropy.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p,
                                              C.c_size_t, C.c_void_p]
+        L.e3_sequence_mean_entropy.restype = C.c_int
+        L.e3_sequence_mean_entropy.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_void_p, C.c_void_p,
+                                               C.c_void_p, C.c_size_t, C.c_void_p]
         L.e3_masked_mean_entropy_static.restype = C.c_int
         L.e3_masked_mean_entropy_static.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p,
                                                     C.c_void_p]
@@ -283,6 +287,26 @@ def e3_masked_mean_entropy(ent, mask=None, out=None, workspace=None, stream=None
     st = lib().e3_masked_mean_entropy(_ptr(ent), _ptr(mask), n, out.data_ptr(), out.data_ptr() + 8,
                                       _ptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream))
     _check("e3_masked_mean_entropy", st)
+    return out
+
+
+def e3_sequence_mean_entropy(ent, mask=None, out=None, workspace=None, stream=None):
+    """Mean over sequences of the per-sequence mean entropy; ``ent`` (and ``mask``) are [n_seq, seq_len].
+    Returns a float64 CUDA tensor [2] = (mean, number of sequences with a token)."""
+    _dev(ent, "ent"); _dev(mask, "mask")
+    if ent.dim() != 2 or ent.dtype != torch.float32 or not ent.is_contiguous():
+        raise ValueError("ent must be a contiguous float32 tensor [n_seq, seq_len]")
+    n_seq, seq_len = ent.shape
+    if mask is not None and (mask.dtype != torch.uint8 or mask.numel() != ent.numel() or not mask.is_contiguous()):
+        raise ValueError("mask must be contiguous uint8 with one entry per token")
+    if out is None:
+        out = torch.empty(2, dtype=torch.float64, device=ent.device)
+    if workspace is None:
+        workspace = torch.empty(e3_workspace_bytes(E3_CALL_SEQUENCE_MEAN_ENTROPY, n_seq), dtype=torch.uint8,
+                                device=ent.device)
+    st = lib().e3_sequence_mean_entropy(_ptr(ent), _ptr(mask), n_seq, seq_len, out.data_ptr(), out.data_ptr() + 8,
+                                        _ptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream))
+    _check("e3_sequence_mean_entropy", st)
     return out
 
 

@@ -48,6 +48,7 @@ extern "C" size_t e3_workspace_bytes(e3_call which, int64_t rows, int64_t V, e3_
     case E3_CALL_TOKEN_LOGP_ENTROPY: return token_mean_offset() + e3::mean_workspace_bytes(rows < 0 ? 0 : rows);
     case E3_CALL_MASKED_MEAN_ENTROPY: return e3::mean_workspace_bytes(rows < 0 ? 0 : rows);
     case E3_CALL_GRPO_OBJECTIVE: return e3::grpo_workspace_bytes(rows);
+    case E3_CALL_SEQUENCE_MEAN_ENTROPY: return e3::seq_mean_workspace_bytes(rows);
   }
   return 0;
 }
@@ -141,6 +142,20 @@ extern "C" e3_status e3_masked_mean_entropy(const float *ent, const uint8_t *mas
   if (!workspace || workspace_bytes < e3::mean_workspace_bytes(n)) return E3_ERR_WORKSPACE;
   cudaError_t e = e3::launch_masked_mean(ent, mask, n, out_mean, out_count, workspace, false,
                                          static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? E3_OK : E3_ERR_CUDA;
+}
+
+extern "C" e3_status e3_sequence_mean_entropy(const float *ent, const uint8_t *mask, int64_t n_seq, int64_t seq_len,
+                                              double *out_mean, double *out_count, void *workspace,
+                                              size_t workspace_bytes, void *stream) {
+  if (n_seq < 0 || seq_len < 0 || n_seq >= (int64_t(1) << 31) || !out_mean || !out_count ||
+      (n_seq > 0 && seq_len > 0 && !ent))
+    return E3_ERR_INVALID_ARG;
+  if (misaligned(ent, 4) || misaligned(out_mean, 8) || misaligned(out_count, 8) || misaligned(workspace, 8))
+    return E3_ERR_ALIGNMENT;
+  if (!workspace || workspace_bytes < e3::seq_mean_workspace_bytes(n_seq)) return E3_ERR_WORKSPACE;
+  cudaError_t e = e3::launch_sequence_mean(ent, mask, n_seq, seq_len, out_mean, out_count, workspace,
+                                           static_cast<cudaStream_t>(stream));
   return e == cudaSuccess ? E3_OK : E3_ERR_CUDA;
 }
 

@@ -75,6 +75,38 @@ __global__ void __launch_bounds__(kMeanThreads) mean_final_kernel(const MeanPart
   }
 }
 
+// Mean of per-sequence means: block s adds the unmasked tokens of sequence s in a fixed order ...
+__global__ void __launch_bounds__(kMeanThreads) seq_partial_kernel(const float *__restrict__ ent,
+                                                                   const uint8_t *__restrict__ mask, int64_t seq_len,
+                                                                   MeanPartial *__restrict__ part) {
+  __shared__ double sh[2 * kMeanThreads / 32];
+  wait_for_stream_predecessor();
+  const int64_t lo = (int64_t)blockIdx.x * seq_len;
+  double s = 0.0, c = 0.0;
+  for (int64_t j = threadIdx.x; j < seq_len; j += kMeanThreads) {
+    const bool on = mask ? mask[lo + j] != 0 : true;
+    if (on) { s += (double)ent[lo + j]; c += 1.0; }
+  }
+  block_reduce_2(s, c, sh);
+  if (threadIdx.x == 0) { part[blockIdx.x].sum = s; part[blockIdx.x].cnt = c; }
+}
+
+// ... and one block averages the sequences' means in index order (sequences without tokens take no part).
+__global__ void __launch_bounds__(kMeanThreads) seq_final_kernel(const MeanPartial *__restrict__ part, int64_t n_seq,
+                                                                 double *__restrict__ out_mean,
+                                                                 double *__restrict__ out_count) {
+  __shared__ double sh[2 * kMeanThreads / 32];
+  wait_for_stream_predecessor();
+  double m = 0.0, c = 0.0;
+  for (int64_t j = threadIdx.x; j < n_seq; j += kMeanThreads)
+    if (part[j].cnt > 0.0) { m += part[j].sum / part[j].cnt; c += 1.0; }
+  block_reduce_2(m, c, sh);
+  if (threadIdx.x == 0) {
+    *out_mean = c > 0.0 ? m / c : CUDART_NAN;
+    *out_count = c;
+  }
+}
+
 // One warp per group; a group of any size is walked in strides of 32.
 __global__ void __launch_bounds__(256) group_advantage_kernel(const float *__restrict__ rewards,
                                                               const int64_t *__restrict__ off, int64_t n_groups,
@@ -148,6 +180,28 @@ cudaError_t launch_masked_mean(const float *ent, const uint8_t *mask, int64_t n,
   cfg.gridDim = dim3(1);
   return cudaLaunchKernelEx(&cfg, mean_final_kernel, (const MeanPartial *)part, blocks, out_mean, out_count,
                             want_sum ? 1 : 0);
+}
+
+size_t seq_mean_workspace_bytes(int64_t n_seq) { return (size_t)(n_seq < 1 ? 1 : n_seq) * sizeof(MeanPartial); }
+
+cudaError_t launch_sequence_mean(const float *ent, const uint8_t *mask, int64_t n_seq, int64_t seq_len,
+                                 double *out_mean, double *out_count, void *workspace, cudaStream_t stream) {
+  MeanPartial *part = static_cast<MeanPartial *>(workspace);
+  cudaLaunchConfig_t cfg = {};
+  cfg.blockDim = dim3(kMeanThreads);
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  if (n_seq > 0) {
+    cfg.gridDim = dim3((unsigned)n_seq);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, seq_partial_kernel, ent, mask, seq_len, part);
+    if (e != cudaSuccess) return e;
+  }
+  cfg.gridDim = dim3(1);
+  return cudaLaunchKernelEx(&cfg, seq_final_kernel, (const MeanPartial *)part, n_seq, out_mean, out_count);
 }
 
 cudaError_t launch_group_advantage(const float *rewards, const int64_t *off, int64_t n_groups, float eps,

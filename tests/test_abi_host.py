@@ -80,6 +80,11 @@ def test_device_calls_reject_bad_arguments_on_the_host(e3):
     assert token(1024, 0, 1, 8, 8, targets=1024, out_ent=1024, out_sum=2052, out_count=2056) == 3
     assert L.e3_masked_mean_entropy(None, None, -1, None, None, None, 0, None) == 1
     assert L.e3_masked_mean_entropy(1024, None, 4, 1024, 1032, None, 0, None) == 4                  # workspace
+    assert L.e3_sequence_mean_entropy(None, None, -1, 4, 1024, 1032, 1024, 64, None) == 1
+    assert L.e3_sequence_mean_entropy(1024, None, 2, 4, None, 1032, 1024, 64, None) == 1
+    assert L.e3_sequence_mean_entropy(1024, None, 2, 4, 1024, 1032, None, 0, None) == 4               # workspace
+    assert L.e3_sequence_mean_entropy(1024, None, 2, 4, 1024, 1032, 1024, 16, None) == 4              # too small
+    assert L.e3_sequence_mean_entropy(1026, None, 2, 4, 1024, 1032, 1024, 64, None) == 3
     assert L.e3_group_advantage(None, None, 0, 1e-6, 1, None, None, None) == 0
     assert L.e3_group_advantage(None, None, 2, 1e-6, 1, None, None, None) == 1
     assert L.e3_group_advantage(None, None, 2, -1.0, 1, None, None, None) == 1                       # eps < 0

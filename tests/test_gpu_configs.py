@@ -57,18 +57,16 @@ def _sample_parity(e3, logits, temps, seed, counter, row_base, sampler, name, ro
 
 
 def _report(name, info):
-    """Parity counts of every configuration: printed (pytest -rP shows them) and kept as one JSON line per
-    case in a file beside the other outputs of a GPU run."""
+    """Parity counts of every configuration: printed (pytest -rP shows them) and, when E3_REPORT_DIR names a
+    directory, appended as one JSON line per case to parity_counts.jsonl there."""
     import json, os
     line = json.dumps({"case": name, **info})
     print("parity:", line)
-    out_dir = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "gpurun_out")
-    try:
+    out_dir = os.environ.get("E3_REPORT_DIR")
+    if out_dir:
         os.makedirs(out_dir, exist_ok=True)
         with open(os.path.join(out_dir, "parity_counts.jsonl"), "a") as f:
             f.write(line + "\n")
-    except OSError:
-        pass
 
 
 @pytest.mark.parametrize("sampler", [0, 1])

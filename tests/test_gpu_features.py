@@ -125,6 +125,33 @@ def test_fused_entropy_sum_feeds_the_scheduler(e3):
     assert e3.e3_update_temperature(s, H_t) == pytest.approx(oracle.update_temperature(so, H_t), rel=1e-12)
 
 
+def test_sequence_mean_entropy_matches_oracle(e3):
+    rng = np.random.default_rng(7)
+    for n_seq, seq_len in ((1, 1), (5, 300), (64, 2048), (300, 33)):
+        ent = torch.from_numpy(rng.random((n_seq, seq_len)).astype(np.float32)).to(DEV)
+        lens = rng.integers(0, seq_len + 1, size=n_seq)
+        mask = torch.from_numpy((np.arange(seq_len)[None, :] < lens[:, None]).astype(np.uint8)).to(DEV)
+        for m in (mask, None):
+            out = e3.e3_sequence_mean_entropy(ent, m)
+            torch.cuda.synchronize()
+            rmean, rused = oracle.sequence_mean_entropy(ent.cpu().numpy(), None if m is None else m.cpu().numpy())
+            assert float(out[1]) == rused
+            if rused == 0:
+                assert math.isnan(float(out[0]))
+            else:
+                assert float(out[0]) == pytest.approx(rmean, rel=1e-12)
+    # the two readings differ when lengths differ
+    e = torch.tensor([[1, 9, 9], [0, 0, 0]], dtype=torch.float32, device=DEV)
+    k = torch.tensor([[1, 0, 0], [1, 1, 1]], dtype=torch.uint8, device=DEV)
+    a = e3.e3_sequence_mean_entropy(e, k)
+    b = e3.e3_masked_mean_entropy(e.reshape(-1), k.reshape(-1))
+    torch.cuda.synchronize()
+    assert a.tolist() == [0.5, 2.0] and b.tolist() == [0.25, 4.0]
+    z = e3.e3_sequence_mean_entropy(torch.zeros((0, 8), device=DEV))
+    torch.cuda.synchronize()
+    assert math.isnan(float(z[0])) and float(z[1]) == 0.0
+
+
 # ----------------------------------------------------------------------------------------------
 # group advantage with eps == 0: identical rewards give 0, not 0/0
 # ----------------------------------------------------------------------------------------------

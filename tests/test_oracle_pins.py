@@ -384,6 +384,29 @@ def test_masked_mean_entropy():
     assert math.isnan(m0) and c0 == 0
 
 
+def test_sequence_mean_entropy_brute_force_and_readings():
+    rng = np.random.default_rng(31)
+    n_seq, seq_len = 9, 37
+    ent = rng.random((n_seq, seq_len)).astype(np.float32)
+    lens = rng.integers(0, seq_len + 1, size=n_seq)
+    lens[2] = 0                                                    # a sequence without tokens takes no part
+    mask = (np.arange(seq_len)[None, :] < lens[:, None]).astype(np.uint8)
+    mean, used = oracle.sequence_mean_entropy(ent, mask)
+    per_seq = [ent[s, :lens[s]].astype(np.float64).mean() for s in range(n_seq) if lens[s] > 0]
+    assert used == len(per_seq) and mean == pytest.approx(float(np.mean(per_seq)), rel=1e-14)
+    # equal lengths (or no mask): the two readings of "average entropy" coincide
+    m2, u2 = oracle.sequence_mean_entropy(ent, None)
+    t2, c2 = oracle.masked_mean_entropy(ent.reshape(-1), None)
+    assert u2 == n_seq and c2 == n_seq * seq_len and m2 == pytest.approx(t2, rel=1e-13)
+    # hand case where they differ: one token of entropy 1, three tokens of entropy 0
+    e = np.array([[1, 9, 9], [0, 0, 0]], np.float32)
+    k = np.array([[1, 0, 0], [1, 1, 1]], np.uint8)
+    assert oracle.sequence_mean_entropy(e, k) == (0.5, 2.0)
+    assert oracle.masked_mean_entropy(e.reshape(-1), k.reshape(-1)) == (0.25, 4.0)
+    nan_mean, zero = oracle.sequence_mean_entropy(e, np.zeros_like(k))
+    assert math.isnan(nan_mean) and zero == 0.0
+
+
 # ----------------------------------------------------------------------------------------------
 # Mean logit gap (App. A: beta sum p_i Delta_i, the first term of H = beta sum p Delta + ln Z)
 # ----------------------------------------------------------------------------------------------
