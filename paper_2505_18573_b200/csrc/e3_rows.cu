@@ -1799,14 +1799,19 @@ __global__ void __launch_bounds__(kThreads, 2) rows_kernel(const __grid_constant
       // describes that use).  A record's buffer comes round again six uses later; by then its bulk store has read it
       // (all but the two most recent stores of this thread have, before a new one is issued).
       const uint32_t rec_lane = ring + kStreamWarps * kNS * kWarpBytes + (uint32_t)lane * kRecordBytesPerWarp;
-      auto ship = [&](uint32_t st, uint32_t par) {
+      auto ship_tile = [&](int64_t ti, uint32_t st, uint32_t par) {
+        bulk_wait_read<2>();
+        bulk_store_s2g(p.ws_records + ti * kRecordFloats, rec_lane + (par * kNS + st) * (uint32_t)(kRecordFloats * 4),
+                       kRecordFloats * 4);
+      };
+      // tile number of the slice the slot's record describes, -1 when it holds no entries (or closes the ring)
+      auto tile_of = [&](uint32_t st) -> int64_t {
         const SliceMeta &pm = sm.meta[lane][st];
-        if (pm.n > 0 && !(pm.flags & kFlagEnd)) {
-          bulk_wait_read<2>();
-          const int64_t ti = pm.row * p.tiles_per_row + pm.s_lo / F::kWarpE;
-          bulk_store_s2g(p.ws_records + ti * kRecordFloats, rec_lane + (par * kNS + st) * (uint32_t)(kRecordFloats * 4),
-                         kRecordFloats * 4);
-        }
+        return (pm.n > 0 && !(pm.flags & kFlagEnd)) ? pm.row * p.tiles_per_row + pm.s_lo / F::kWarpE : (int64_t)-1;
+      };
+      auto ship = [&](uint32_t st, uint32_t par) {
+        const int64_t ti = tile_of(st);
+        if (ti >= 0) ship_tile(ti, st, par);
       };
       unsigned long long idle_since = 0;         // 0: the last pass over the lanes fed something
       uint32_t idle_passes = 0;
@@ -1822,8 +1827,11 @@ __global__ void __launch_bounds__(kThreads, 2) rows_kernel(const __grid_constant
             ready = ok != 0;
           }
           if (ready) {
-            if (SAMPLER == 1 && issued >= (uint32_t)kNS) ship(slot, phase);
+            // sampler 1: the record of the slot's previous use goes out AFTER the refill has been issued (the refill
+            // is what the consumer warp waits for); its slice is read from the slot's record before that is rewritten
+            const int64_t prev_tile = (SAMPLER == 1 && issued >= (uint32_t)kNS) ? tile_of(slot) : (int64_t)-1;
             feeder.feed(p, sm, ring_w, lane, (int)slot);
+            if (SAMPLER == 1 && prev_tile >= 0) ship_tile(prev_tile, slot, phase);
             if (!feeder.stalled) {
               ++issued;
               if (++slot == kNS) { slot = 0; phase ^= 1u; }
