@@ -316,3 +316,22 @@ def test_closed_loop_entropy_scaling_with_alpha(e3):
             assert abs(math.log(ratio)) <= abs(math.log(alpha)) * 1.6, (alpha, name, ratio)
         assert abs(math.log(report[(alpha, "surrogate")])) > 0.02 * abs(math.log(alpha))
     print("closed loop H1/H0:", {f"alpha={a} {n}": round(v, 4) for (a, n), v in report.items()})
+
+
+# ----------------------------------------------------------------------------------------------
+# measurement aid: the read-only probe really reads every word once
+# ----------------------------------------------------------------------------------------------
+def test_probe_read_checksum(e3):
+    rng = np.random.default_rng(3)
+    for n_words in (4, 4 * 1000, 4 * 123457):       # multiples of 16 bytes, smaller and larger than one pass of the grid
+        host = rng.integers(0, 1 << 32, size=n_words, dtype=np.uint64).astype(np.uint32)
+        buf = torch.from_numpy(host.view(np.int32)).to(DEV)
+        scratch = torch.zeros(e3.E3_PROBE_SCRATCH_BYTES, dtype=torch.uint8, device=DEV)
+        e3.e3_probe_read(buf, scratch=scratch)
+        torch.cuda.synchronize()
+        per_cta = scratch.cpu().numpy().view(np.uint64)
+        v = host.reshape(-1, 4).astype(np.uint64)
+        want = int(((v[:, 0] ^ v[:, 1]) + (v[:, 2] ^ v[:, 3])).sum() % (1 << 32))
+        assert int(per_cta.sum() % (1 << 32)) == want
+    with pytest.raises(e3.E3Error):
+        e3.e3_probe_read(torch.zeros(3, dtype=torch.int32, device=DEV))     # not a multiple of 16 bytes
