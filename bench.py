@@ -50,7 +50,7 @@ METRIC = "logit rows/s, fused sample+entropy, V=151,936"
 UNIT = "rows/s"
 # dram__bytes_read.sum + dram__bytes_write.sum of one e3_sample launch of this workload (ncu capture summarised in
 # profiles/rows_kernel_c2_ncu_full.txt and rows_kernel_sampler0_c2_ncu_full.txt), streaming kernel only.
-NCU_TRAFFIC_BYTES = {0: 161.7e6, 1: 160.2e6}
+NCU_TRAFFIC_BYTES = {0: 161.7e6, 1: 160.0e6}
 WORKLOAD = "rollout decode step: 512 rows (64 prompts x 8 rollouts) x V=151,936 bf16, 256 decode steps"
 
 
